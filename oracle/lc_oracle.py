@@ -1,0 +1,144 @@
+"""ctypes binding of the C++ CPU oracle (``lc_oracle.cpp``).
+
+Test infrastructure only: the tests, the smoke check and the benchmark's CPU-baseline leg use it to
+check and to time the method as the paper states it. The CUDA library never imports this module.
+All arrays are numpy arrays in host memory.
+"""
+import ctypes as C
+
+import numpy as np
+
+from . import build as _build
+
+OK, ERR_ARG, ERR_CAPACITY, ERR_NONFINITE, ERR_FORMAT, ERR_MISMATCH = 0, -1, -2, -3, -4, -5
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(_build.build())
+        u64, i32, vp = C.c_uint64, C.c_int, C.c_void_p
+        L.lco_bins.argtypes = [vp, vp, u64, vp, vp, vp]
+        L.lco_table.argtypes = [vp, vp, u64, i32, vp, vp, vp, vp, vp]
+        L.lco_symbols.argtypes = [vp, vp, u64, i32, vp]
+        L.lco_huffman.argtypes = [vp, i32, vp, vp]
+        L.lco_midrange.argtypes = [C.c_float, C.c_float]
+        L.lco_midrange.restype = C.c_float
+        L.lco_model_bits.argtypes = [u64, u64, u64]
+        L.lco_model_bits.restype = u64
+        L.lco_stream_bound.argtypes = [u64, i32]
+        L.lco_stream_bound.restype = u64
+        L.lco_compress.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64)]
+        L.lco_decode_symbols.argtypes = [vp, u64, u64, vp]
+        L.lco_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp]
+        _lib = L
+    return _lib
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code):
+        super().__init__("oracle status %d" % code)
+        self.code = code
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a, a.ctypes.data
+
+
+def bins(base, cur):
+    """(count[512] u64, mmin[512] u32, mmax[512] u32) of the delta's (sign, exponent) buckets."""
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    count = np.zeros(512, np.uint64)
+    mmin = np.zeros(512, np.uint32)
+    mmax = np.zeros(512, np.uint32)
+    lib().lco_bins(pb, pc, base.size, count.ctypes.data, mmin.ctypes.data, mmax.ctypes.data)
+    return count, mmin, mmax
+
+
+def table(base, cur, nbits):
+    """dict(key, rep, count, len, code), each of length nsym."""
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    key = np.zeros(256, np.int32)
+    rep = np.zeros(256, np.float32)
+    count = np.zeros(256, np.uint64)
+    ln = np.zeros(256, np.int32)
+    code = np.zeros(256, np.uint64)
+    rc = lib().lco_table(pb, pc, base.size, nbits, key.ctypes.data, rep.ctypes.data, count.ctypes.data,
+                         ln.ctypes.data, code.ctypes.data)
+    if rc < 0:
+        raise OracleError(rc)
+    return dict(key=key[:rc], rep=rep[:rc], count=count[:rc], len=ln[:rc], code=code[:rc])
+
+
+def symbols(base, cur, nbits):
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    sym = np.zeros(base.size, np.uint8)
+    rc = lib().lco_symbols(pb, pc, base.size, nbits, sym.ctypes.data)
+    if rc < 0:
+        raise OracleError(rc)
+    return sym
+
+
+def huffman(count):
+    count = np.ascontiguousarray(count, dtype=np.uint64)
+    ln = np.zeros(count.size, np.int32)
+    code = np.zeros(count.size, np.uint64)
+    rc = lib().lco_huffman(count.ctypes.data, count.size, ln.ctypes.data, code.ctypes.data)
+    if rc < 0:
+        raise OracleError(rc)
+    return ln, code
+
+
+def midrange(vmin, vmax):
+    return np.float32(lib().lco_midrange(float(np.float32(vmin)), float(np.float32(vmax))))
+
+
+def model_bits(n, k, b=32):
+    return int(lib().lco_model_bits(n, k, b))
+
+
+def stream_bound(n, nbits):
+    return int(lib().lco_stream_bound(n, nbits))
+
+
+def compress(base, cur, nbits):
+    """Returns the stream as a uint8 numpy array."""
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    if not 1 <= nbits <= 8:
+        raise OracleError(ERR_ARG)
+    cap = stream_bound(base.size, nbits)
+    buf = np.zeros(cap, np.uint8)
+    out = C.c_uint64(0)
+    rc = lib().lco_compress(pb, pc, base.size, nbits, buf.ctypes.data, cap, C.byref(out))
+    if rc < 0:
+        raise OracleError(rc)
+    return buf[: out.value].copy()
+
+
+def decode_symbols(stream, n):
+    stream = np.ascontiguousarray(stream, dtype=np.uint8)
+    sym = np.zeros(n, np.uint8)
+    rc = lib().lco_decode_symbols(stream.ctypes.data, stream.size, n, sym.ctypes.data)
+    if rc < 0:
+        raise OracleError(rc)
+    return sym
+
+
+def recover(base, streams):
+    base, pb = _f32(base)
+    streams = [np.ascontiguousarray(s, dtype=np.uint8) for s in streams]
+    k = len(streams)
+    ptrs = (C.c_void_p * k)(*[s.ctypes.data for s in streams])
+    sizes = (C.c_uint64 * k)(*[s.size for s in streams])
+    out = np.zeros(base.size, np.float32)
+    rc = lib().lco_recover(pb, ptrs, sizes, k, base.size, out.ctypes.data)
+    if rc < 0:
+        raise OracleError(rc)
+    return out

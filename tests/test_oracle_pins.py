@@ -1,0 +1,441 @@
+"""Pins of the CPU oracle to facts fixed by the paper and by mathematics (CPU only).
+
+Each test is chosen so that a plausible mistake in one step of the oracle (a dropped term, a wrong
+sign, index, order or rounding) fails it. Nothing here calls the CUDA path.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+from conftest import load_golden
+
+
+def f32(bits):
+    return np.array(bits, np.uint32).view(np.float32)
+
+
+# ---------------------------------------------------------------- hand-worked golden streams
+
+
+@pytest.mark.parametrize("name", ["ten_elements_nbits2.txt", "skew16_nbits3.txt"])
+def test_golden_stream_bytes(oracle, name):
+    g = load_golden(name)
+    base = np.zeros(g["cur"].size, np.float32)
+    s = oracle.compress(base, g["cur"], g["nbits"])
+    assert s.tobytes() == g["stream"].tobytes()
+    out = oracle.recover(base, [g["stream"]])
+    assert out.view(np.uint32).tolist() == g["recovered"].view(np.uint32).tolist()
+
+
+def test_paper_size_model_example(oracle):
+    # Section 3.1.1 worked example: n = 10, b = 32, k = 5 -> 190 bits, rate 1.68.
+    bits = oracle.model_bits(10, 5, 32)
+    assert bits == 190
+    assert round(10 * 32 / bits, 2) == 1.68
+    # and the 2-bit promotion of that example leaves 4 buckets of 2 bits each.
+    assert oracle.model_bits(10, 4, 32) == 10 * 2 + 4 * 32
+
+
+def test_paper_example_shape(oracle):
+    # Figure 1 text: 10 elements, 5 buckets; 2-bit promotion keeps 3 and merges 2 into the zero bucket.
+    g = load_golden("ten_elements_nbits2.txt")
+    base = np.zeros(10, np.float32)
+    count, _, _ = oracle.bins(base, g["cur"])
+    assert int((count > 0).sum()) == 5
+    t = oracle.table(base, g["cur"], 2)
+    assert len(t["key"]) == 4 and t["rep"][0] == 0.0 and int(t["count"][0]) == 2
+
+
+# ---------------------------------------------------------------- O1-O3: delta and buckets
+
+
+def test_bins_hand_vector(oracle):
+    # known bit patterns: 1.0, 1.5, -0.75, smallest normal, a subnormal, +0, -0, and a delta that is
+    # only representable after the fp32 subtract rounds.
+    cur = f32([0x3F800000, 0x3FC00000, 0xBF400000, 0x00800000, 0x00000001, 0x00000000, 0x80000000])
+    base = np.zeros(cur.size, np.float32)
+    count, mmin, mmax = oracle.bins(base, cur)
+    exp = {127: 2, 256 + 126: 1, 1: 1, 0: 2, 256: 1}
+    for key in range(512):
+        assert int(count[key]) == exp.get(key, 0), key
+    assert (mmin[127], mmax[127]) == (0, 0x400000)
+    assert (mmin[256 + 126], mmax[256 + 126]) == (0x400000, 0x400000)
+    assert (mmin[0], mmax[0]) == (0, 1)  # +0 and the subnormal share E = 0, s = 0
+
+
+def test_delta_is_fp32_subtract(oracle):
+    # cur - base must be rounded once to fp32: 1 + 2^-24 is not representable, and (1+2^-23) - 2^-24
+    # rounds to even.
+    base = np.array([np.float32(2.0 ** -24)], np.float32)
+    cur = f32([0x3F800001])
+    d = (cur - base).view(np.uint32)[0]
+    count, mmin, mmax = oracle.bins(base, cur)
+    key = int(d >> 23)
+    assert count[key] == 1 and mmin[key] == (d & 0x7FFFFF) == mmax[key]
+
+
+def test_bins_against_sort_and_group(oracle):
+    rng = np.random.default_rng(5)
+    n = 20011
+    base = rng.normal(0, 0.02, n).astype(np.float32)
+    cur = (base + rng.laplace(0, 1e-3, n).astype(np.float32)).astype(np.float32)
+    cur[::97] = base[::97]  # exact zeros
+    count, mmin, mmax = oracle.bins(base, cur)
+    bits = (cur - base).view(np.uint32)
+    order = np.sort(bits)
+    keys = order >> 23
+    assert int(count.sum()) == n
+    for key in np.unique(keys):
+        grp = order[keys == key]
+        assert int(count[key]) == grp.size
+        assert int(mmin[key]) == int(grp[0] & 0x7FFFFF)
+        assert int(mmax[key]) == int(grp[-1] & 0x7FFFFF)
+    assert all(count[k] == 0 for k in range(512) if k not in set(keys.tolist()))
+
+
+# ---------------------------------------------------------------- O4: priority promotion
+
+
+def _vector_with_keys(keys):
+    """One element per (s, E) key, mantissa 0."""
+    bits = [((k >> 8) << 31) | ((k & 255) << 23) for k in keys]
+    return f32(bits)
+
+
+def test_selection_order_and_limit(oracle):
+    keys = [100, 256 + 100, 130, 256 + 131, 90, 256 + 90, 1, 254, 0, 256]  # includes E=0 keys
+    cur = _vector_with_keys(keys)
+    base = np.zeros(cur.size, np.float32)
+    full = [254, 256 + 131, 130, 100, 256 + 100, 90, 256 + 90, 1]  # E desc, + before -
+    for nbits in range(1, 9):
+        t = oracle.table(base, cur, nbits)
+        K = min(2 ** nbits - 1, len(full))
+        assert t["key"].tolist() == [0] + full[:K]
+        assert len(t["key"]) <= 2 ** nbits
+        assert int(t["count"][0]) == len(keys) - K
+        sym = oracle.symbols(base, cur, nbits)
+        for i, k in enumerate(keys):
+            assert sym[i] == (full.index(k) + 1 if k in full[:K] else 0)
+
+
+def test_subnormals_and_zero_never_selected(oracle):
+    cur = f32([0x00000001, 0x807FFFFF, 0x00000000, 0x80000000])
+    t = oracle.table(np.zeros(4, np.float32), cur, 8)
+    assert t["key"].tolist() == [0] and int(t["count"][0]) == 4 and t["len"].tolist() == [0]
+
+
+def test_nonfinite_rejected(oracle):
+    for bad in (0x7F800000, 0xFF800000, 0x7FC00000):
+        cur = f32([0x3F800000, bad])
+        with pytest.raises(oracle.OracleError) as e:
+            oracle.compress(np.zeros(2, np.float32), cur, 4)
+        assert e.value.code == oracle.ERR_NONFINITE
+
+
+# ---------------------------------------------------------------- O5: representative
+
+
+def _int_midrange(s, E, m0, m1):
+    t = m0 + m1
+    mr = t >> 1
+    if (t & 1) and (mr & 1):
+        mr += 1
+    return (s << 31) | (E << 23) | mr
+
+
+def test_midrange_equals_integer_formula(oracle):
+    rng = np.random.default_rng(11)
+    cases = [(0, 254, 0x7FFFFE, 0x7FFFFF), (1, 254, 0x7FFFFF, 0x7FFFFF), (0, 1, 0, 1), (1, 1, 1, 2),
+             (0, 127, 1, 2), (0, 127, 1, 4), (0, 127, 3, 4), (0, 127, 0x7FFFFD, 0x7FFFFE)]
+    for _ in range(4000):
+        m0, m1 = sorted(rng.integers(0, 1 << 23, 2).tolist())
+        cases.append((int(rng.integers(0, 2)), int(rng.integers(1, 255)), m0, m1))
+    for s, E, m0, m1 in cases:
+        lo = f32([(s << 31) | (E << 23) | m0])[0]
+        hi = f32([(s << 31) | (E << 23) | m1])[0]
+        vmin, vmax = (hi, lo) if s else (lo, hi)
+        rep = oracle.midrange(vmin, vmax)
+        assert int(np.float32(rep).view(np.uint32)) == _int_midrange(s, E, m0, m1), (s, E, m0, m1)
+        assert vmin <= rep <= vmax
+
+
+def test_rep_single_element_bucket_is_the_element(oracle):
+    cur = f32([0x3DCCCCCD, 0xBDCCCCCD, 0x3A83126F])
+    t = oracle.table(np.zeros(3, np.float32), cur, 4)
+    assert sorted(t["rep"][1:].view(np.uint32).tolist()) == sorted(cur.view(np.uint32).tolist())
+
+
+# ---------------------------------------------------------------- O6: Huffman
+
+
+def _brute_force_cost(counts, max_len):
+    best = None
+    for lens in itertools.product(range(1, max_len + 1), repeat=len(counts)):
+        if sum(2.0 ** -l for l in lens) <= 1.0 + 1e-12:
+            cost = sum(c * l for c, l in zip(counts, lens))
+            best = cost if best is None else min(best, cost)
+    return best
+
+
+def test_huffman_optimal_vs_brute_force(oracle):
+    rng = np.random.default_rng(3)
+    trials = []
+    for k in range(2, 7):
+        for _ in range(12):
+            trials.append(rng.integers(1, 40, k).tolist())        # random
+            trials.append(rng.integers(1, 4, k).tolist())         # tie-heavy
+        trials.append([1] * k)
+        trials.append([2 ** i for i in range(k)])
+    for counts in trials:
+        ln, code = oracle.huffman(counts)
+        cost = sum(c * int(l) for c, l in zip(counts, ln))
+        assert cost == _brute_force_cost(counts, len(counts)), counts
+
+
+def _kraft_and_prefix_free(ln, code):
+    used = [(int(l), int(c)) for l, c in zip(ln, code) if l > 0]
+    assert sum(2 ** (64 - l) for l, _ in used) == 2 ** 64  # Kraft equality, exact
+    strs = [format(c, "0%db" % l) for l, c in used]
+    for a, b in itertools.permutations(strs, 2):
+        assert not b.startswith(a)
+
+
+def test_huffman_kraft_entropy_prefix(oracle):
+    rng = np.random.default_rng(4)
+    for k in (2, 3, 5, 8, 16, 31, 32, 64, 200, 256):
+        for scale in (1.0, 1e3, 1e9):
+            counts = np.maximum(1, (rng.pareto(1.2, k) * scale).astype(np.uint64))
+            ln, code = oracle.huffman(counts)
+            _kraft_and_prefix_free(ln, code)
+            p = counts / counts.sum()
+            H = float(-(p * np.log2(p)).sum())
+            Lbar = float((p * ln).sum())
+            assert H - 1e-9 <= Lbar < H + 1
+
+
+def test_huffman_textbook_cases(oracle):
+    for j in range(1, 9):  # 2^j equal counts -> all lengths j
+        ln, _ = oracle.huffman([7] * (2 ** j))
+        assert ln.tolist() == [j] * (2 ** j)
+    ln, _ = oracle.huffman([1, 1, 2, 4, 8, 16])  # dyadic
+    assert ln.tolist() == [5, 5, 4, 3, 2, 1]
+    fib = [1, 1, 2, 3, 5, 8, 13, 21, 34, 55, 89, 144]  # maximal depth
+    ln, _ = oracle.huffman(fib)
+    assert ln.tolist() == [11, 11, 10, 9, 8, 7, 6, 5, 4, 3, 2, 1]
+    big = [1, 1]
+    while len(big) < 45:
+        big.append(big[-1] + big[-2])
+    ln, code = oracle.huffman(big)  # total < 2^32, depth 44: codes longer than 32 bits
+    assert int(ln.max()) == 44 and sum(big) < 2 ** 32
+    _kraft_and_prefix_free(ln, code)
+
+
+def test_huffman_tie_break_and_canonical_hand_case(oracle):
+    # five equal counts, worked by hand with the two-queue rule (leaf before internal node on ties):
+    # (a+b)=2, (c+d)=2, e+(ab)=3, (cd)+3=5 -> a,b depth 3; c,d,e depth 2.
+    ln, code = oracle.huffman([1, 1, 1, 1, 1])
+    assert ln.tolist() == [3, 3, 2, 2, 2]
+    assert code.tolist() == [0b110, 0b111, 0b00, 0b01, 0b10]
+    # zero-count symbols take no part and get length 0
+    ln, code = oracle.huffman([0, 5, 0, 5, 0])
+    assert ln.tolist() == [0, 1, 0, 1, 0] and code.tolist() == [0, 0, 0, 1, 0]
+    # one used symbol -> length 0
+    ln, _ = oracle.huffman([0, 9, 0])
+    assert ln.tolist() == [0, 0, 0]
+
+
+def test_canonical_codes_increase(oracle):
+    rng = np.random.default_rng(8)
+    counts = rng.integers(1, 10 ** 6, 100)
+    ln, code = oracle.huffman(counts)
+    order = sorted(range(100), key=lambda j: (ln[j], j))
+    vals = [int(code[j]) << (int(ln.max()) - int(ln[j])) for j in order]  # left-aligned
+    assert all(a < b for a, b in zip(vals, vals[1:]))
+
+
+# ---------------------------------------------------------------- O7: stream
+
+
+def _random_case(rng, n, scale=1e-3):
+    base = rng.normal(0, 0.02, n).astype(np.float32)
+    cur = (base + rng.laplace(0, scale, n).astype(np.float32)).astype(np.float32)
+    return base, cur
+
+
+@pytest.mark.parametrize("n", [0, 1, 3, 4, 5, 127, 128, 129, 4095, 4096, 4097, 3 * 4096 + 77, 70001])
+@pytest.mark.parametrize("nbits", [1, 3, 8])
+def test_roundtrip_symbols_and_sizes(oracle, n, nbits):
+    rng = np.random.default_rng(n * 10 + nbits)
+    base, cur = _random_case(rng, n)
+    s = oracle.compress(base, cur, nbits)
+    assert s.size <= oracle.stream_bound(n, nbits)
+    t = oracle.table(base, cur, nbits)
+    sym = oracle.symbols(base, cur, nbits)
+    assert np.array_equal(oracle.decode_symbols(s, n), sym)
+    # header fields
+    payload_bits = int(np.frombuffer(s[40:48].tobytes(), "<u8")[0])
+    assert payload_bits == int((t["count"] * t["len"].astype(np.uint64)).sum())
+    assert int(np.frombuffer(s[48:56].tobytes(), "<u8")[0]) == s.size
+    nchunks = (n + 4095) // 4096
+    nsym = len(t["key"])
+    ci = 64 + 16 * nsym
+    li = ci + 8 * (nchunks + 1)
+    chunk_off = np.frombuffer(s[ci:li].tobytes(), "<u8")
+    lane_bits = np.frombuffer(s[li:li + 64 * nchunks].tobytes(), "<u2").reshape(nchunks, 32)
+    assert int(lane_bits.sum()) == payload_bits
+    sizes = np.diff(chunk_off)
+    assert np.array_equal(sizes, ((lane_bits.sum(1).astype(np.int64) + 7) // 8 + 15) // 16 * 16)
+    # lane lengths recomputed from the symbols and the element order of the format
+    ln = t["len"]
+    for c in range(nchunks):
+        for lane in (0, 1, 31):
+            idx = [4096 * c + 128 * j + 4 * lane + e for j in range(32) for e in range(4)]
+            idx = [i for i in idx if i < n]
+            assert int(lane_bits[c, lane]) == int(sum(int(ln[sym[i]]) for i in idx))
+
+
+def test_payload_bits_by_independent_bit_writer(oracle):
+    # re-create one chunk's payload from (symbols, codes) with python string concatenation.
+    rng = np.random.default_rng(21)
+    n = 4096 + 600
+    base, cur = _random_case(rng, n)
+    s = oracle.compress(base, cur, 4)
+    t = oracle.table(base, cur, 4)
+    sym = oracle.symbols(base, cur, 4)
+    nsym, nchunks = len(t["key"]), 2
+    ci = 64 + 16 * nsym
+    li = ci + 8 * (nchunks + 1)
+    po = (li + 64 * nchunks + 15) // 16 * 16
+    chunk_off = np.frombuffer(s[ci:li].tobytes(), "<u8")
+    for c in range(nchunks):
+        bits = ""
+        for lane in range(32):
+            for j in range(32):
+                for e in range(4):
+                    i = 4096 * c + 128 * j + 4 * lane + e
+                    if i < n and t["len"][sym[i]] > 0:
+                        bits += format(int(t["code"][sym[i]]), "0%db" % int(t["len"][sym[i]]))
+        nbytes = ((len(bits) + 7) // 8 + 15) // 16 * 16
+        bits = bits.ljust(nbytes * 8, "0")
+        words = [int(bits[w:w + 32], 2) for w in range(0, len(bits), 32)]
+        expect = np.array(words, "<u4").tobytes()
+        got = s[po + int(chunk_off[c]): po + int(chunk_off[c + 1])].tobytes()
+        assert got == expect
+
+
+def test_single_symbol_and_empty(oracle):
+    base = np.linspace(-1, 1, 5000).astype(np.float32)
+    s = oracle.compress(base, base, 5)  # all-zero delta
+    assert int(np.frombuffer(s[40:48].tobytes(), "<u8")[0]) == 0  # no payload bits
+    assert s[20] == 0  # max_len
+    out = oracle.recover(base, [s])
+    assert np.array_equal(out.view(np.uint32), (base + np.float32(0)).view(np.uint32))
+    # one exponent, one sign, no zeros: the single used symbol is symbol 1
+    cur = (1.0 + np.random.default_rng(0).random(3000)).astype(np.float32)
+    s = oracle.compress(np.zeros(3000, np.float32), cur, 2)
+    assert np.all(oracle.decode_symbols(s, 3000) == 1)
+    s0 = oracle.compress(np.zeros(0, np.float32), np.zeros(0, np.float32), 3)
+    assert s0.size == 64 + 16 + 8 + 8  # header, one table entry, chunk_off[0], padding to 16
+    assert oracle.recover(np.zeros(0, np.float32), [s0]).size == 0
+
+
+# ---------------------------------------------------------------- O8: recovery
+
+
+def test_recover_equals_base_plus_rep(oracle):
+    rng = np.random.default_rng(31)
+    n = 30000
+    base, cur = _random_case(rng, n)
+    base[:5] = f32([0x80000000] * 5)  # -0.0 base: adding the +0 representative gives +0.0
+    cur[:5] = base[:5]
+    for nbits in (2, 4, 6):
+        s = oracle.compress(base, cur, nbits)
+        t = oracle.table(base, cur, nbits)
+        sym = oracle.symbols(base, cur, nbits)
+        expect = base + t["rep"][sym]
+        out = oracle.recover(base, [s])
+        assert np.array_equal(out.view(np.uint32), expect.view(np.uint32))
+        assert out[:5].view(np.uint32).tolist() == [0] * 5
+        # error bound of exponent quantization: kept elements stay within half a binade's width
+        d = cur - base
+        dq = t["rep"][sym]
+        kept = sym > 0
+        e = np.floor(np.log2(np.abs(d[kept])))
+        assert np.all(np.abs(dq[kept].astype(np.float64) - d[kept]) < 2.0 ** (e - 1) + 1e-300)
+        assert np.all(dq[~kept] == 0)
+        assert np.all(np.sign(dq[kept]) == np.sign(d[kept]))
+
+
+def test_chain_identity(oracle):
+    # Algorithm 1: tracked state u~_t = u~_{t-1} + quantized delta; recovery from u_0 and all streams
+    # reproduces u~_t bit for bit.
+    rng = np.random.default_rng(41)
+    n = 9001
+    u0 = rng.normal(0, 0.05, n).astype(np.float32)
+    u, tracked, streams = u0.copy(), u0.copy(), []
+    for t in range(5):
+        u = (u + rng.normal(0, 1e-3, n).astype(np.float32)).astype(np.float32)
+        s = oracle.compress(tracked, u, 3)
+        streams.append(s)
+        tracked = oracle.recover(tracked, [s])
+        out = oracle.recover(u0, streams)
+        assert np.array_equal(out.view(np.uint32), tracked.view(np.uint32))
+    # error feedback keeps the tracked state near the true state
+    assert float(np.abs(tracked - u).max()) < 5e-3
+
+
+def test_compress_of_identical_states(oracle):
+    x = np.random.default_rng(2).normal(0, 1, 10000).astype(np.float32)
+    s = oracle.compress(x, x, 4)
+    assert np.all(oracle.decode_symbols(s, x.size) == 0)
+
+
+# ---------------------------------------------------------------- malformed streams
+
+
+def test_reader_rejects_corruption(oracle):
+    rng = np.random.default_rng(51)
+    n = 10000
+    base, cur = _random_case(rng, n)
+    good = oracle.compress(base, cur, 4)
+    assert oracle.recover(base, [good]).size == n
+
+    def expect(mut, code):
+        bad = good.copy()
+        mut(bad)
+        with pytest.raises(oracle.OracleError) as e:
+            oracle.recover(base, [bad])
+        assert e.value.code == code
+
+    def setb(off, val):
+        return lambda b: b.__setitem__(off, val)
+
+    expect(setb(0, ord("X")), oracle.ERR_FORMAT)     # magic
+    expect(setb(4, 2), oracle.ERR_FORMAT)            # version
+    expect(setb(6, 9), oracle.ERR_FORMAT)            # nbits
+    expect(setb(16, 200), oracle.ERR_FORMAT)         # nsym > 2^nbits
+    expect(setb(24, 1), oracle.ERR_FORMAT)           # chunk_elems
+    expect(setb(64 + 16 + 2, 1), oracle.ERR_FORMAT)  # a code length changed: Kraft / payload_bits
+    expect(setb(48, (int(good[48]) + 16) % 256), oracle.ERR_FORMAT)  # total_bytes
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.recover(base, [good[:-16]])           # truncated buffer
+    assert e.value.code == oracle.ERR_FORMAT
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.recover(base[:-1], [good])
+    assert e.value.code == oracle.ERR_MISMATCH
+
+
+def test_ratio_ranges_on_synthetic_deltas(oracle):
+    # Section 4.3 reports E+P+H below 5 % (2-bit) and 10 % (3-bit) on its training deltas; a
+    # concentrated synthetic delta must land in the same region (sanity range, not an acceptance test).
+    rng = np.random.default_rng(61)
+    n = 200000
+    base = rng.normal(0, 0.02, n).astype(np.float32)
+    cur = (base + rng.normal(0, 1e-3, n).astype(np.float32)).astype(np.float32)
+    for nbits, limit in ((2, 0.05), (3, 0.10)):
+        s = oracle.compress(base, cur, nbits)
+        payload_bits = int(np.frombuffer(s[40:48].tobytes(), "<u8")[0])
+        assert payload_bits / (32 * n) < limit
+        assert payload_bits <= n * nbits
