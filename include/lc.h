@@ -1,0 +1,144 @@
+/*
+ * lc.h - C ABI of the LC-Checkpoint compress / recover library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the per-snapshot compress pass and the recovery pass of the lossy
+ * delta-encoding checkpoint scheme of "On Efficient Constructions of Checkpoints" (arxiv 2009.13003):
+ * Algorithm 1 steps 4-7, Section 3.1.1 (exponent-based quantization, priority promotion, midrange
+ * representative) and Section 3.1.2 (Huffman coding), and the reconstruction identity
+ * u_t = u_0 + sum of the quantized deltas (Section 3, after component C2).
+ *
+ * Conventions for every call
+ *  - Pointers marked DEVICE are CUDA device pointers owned by the caller; pointers marked HOST are
+ *    ordinary host pointers. The library allocates no memory and keeps no state between calls.
+ *  - Work is enqueued on the CUDA stream `cs` (0 = the default stream) and, unless stated, the call
+ *    returns without waiting for it. Buffers must stay valid until that work has finished.
+ *  - Return value: LC_OK (0) or a negative LC_ERR_* code. Errors that only the device can see
+ *    (non-finite delta, malformed stream, a bounded wait that gave up) are written to a status word
+ *    in the workspace and read back with lc_last_status(). No call aborts, throws or traps.
+ *  - The byte format of a stream is fixed by docs/FORMAT.md, version 1.
+ */
+#ifndef LC_H_
+#define LC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LC_OK 0
+#define LC_ERR_ARG (-1)       /* null / misaligned pointer, nbits outside 1..8, k outside 1..LC_MAX_CHAIN, n >= 2^32 */
+#define LC_ERR_CAPACITY (-2)  /* stream or workspace buffer too small */
+#define LC_ERR_NONFINITE (-3) /* some delta is Inf or NaN; the stream must not be used */
+#define LC_ERR_FORMAT (-4)    /* malformed stream */
+#define LC_ERR_MISMATCH (-5)  /* a stream's element count differs from n */
+#define LC_ERR_TIMEOUT (-6)   /* a bounded device-side wait gave up */
+#define LC_ERR_CUDA (-7)      /* a CUDA runtime call failed */
+
+#define LC_MAX_CHAIN 8 /* most streams one lc_recover call applies */
+
+/* Same underlying type as cudaStream_t, so a cudaStream_t can be passed directly. */
+typedef struct CUstream_st* lc_cuda_stream_t;
+
+/* Host copy of a stream header (format section 3.1). */
+typedef struct lc_info {
+  uint64_t n;              /* elements */
+  uint64_t total_bytes;    /* size of the whole stream */
+  uint64_t payload_bits;   /* sum of code lengths */
+  uint64_t payload_offset; /* byte offset of the payload */
+  uint32_t nbits;          /* bits of priority promotion */
+  uint32_t nsym;           /* kept buckets + 1 */
+  uint32_t max_len;        /* longest code */
+  uint32_t nchunks;
+  int32_t valid;           /* 1 if magic, version and constants are those of format version 1 */
+} lc_info;
+
+/* Library version (major*100 + minor). */
+int lc_version(void);
+
+/* Static text for a status code. */
+const char* lc_strerror(int code);
+
+/* Upper bound in bytes of the stream lc_compress writes for n elements (format section 6). Holds
+ * because a Huffman code never uses more bits in total than the fixed nbits-bit code. */
+uint64_t lc_stream_bound(uint64_t n, int nbits);
+
+/* Bytes of DEVICE scratch lc_compress and lc_recover need for vectors of up to n elements. */
+uint64_t lc_workspace_bytes(uint64_t n);
+
+/*
+ * Compress pass (Algorithm 1 steps 4-6; Sections 3.1.1-3.1.2).
+ *   stream <- LC(cur - base): the fp32 delta of `cur` against the tracked state `base` is bucketed by
+ *   sign and exponent, the 2^nbits - 1 occupied buckets with the largest exponent are kept and
+ *   represented by the midrange of their values, everything else becomes zero, and the bucket symbols
+ *   are Huffman-coded.
+ * base, cur   DEVICE, read-only, n contiguous fp32 each, 16-byte aligned.
+ * n           number of elements, 0 <= n < 2^32.
+ * nbits       x of the x-bit priority promotion, 1..8.
+ * stream      DEVICE, written; 16-byte aligned; stream_capacity >= lc_stream_bound(n, nbits).
+ *             The stream's size is in its header (lc_stream_info).
+ * workspace   DEVICE scratch, 256-byte aligned, workspace_bytes >= lc_workspace_bytes(n). Its contents
+ *             are overwritten; two calls that overlap in time need two workspaces.
+ * Host-detectable errors return at once (LC_ERR_ARG, LC_ERR_CAPACITY, LC_ERR_CUDA). A delta with
+ * exponent field 255 sets LC_ERR_NONFINITE in the status word and leaves the stream without its magic.
+ */
+int lc_compress(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs);
+
+/*
+ * Recovery pass (Algorithm 1 step 7 applied k times; u_t = u_0 + sum_i quantized delta_i).
+ *   out_i = fl32(...fl32(fl32(base_i + d_0,i) + d_1,i)... + d_{k-1},i), streams applied in array order.
+ * base          DEVICE, n fp32, 16-byte aligned.
+ * streams       HOST array of k DEVICE pointers (16-byte aligned) to streams written by lc_compress.
+ * stream_bytes  HOST array of k buffer sizes in bytes; no byte beyond them is read.
+ * k             1..LC_MAX_CHAIN.
+ * n             elements in base and out; every stream's header must say the same n.
+ * out           DEVICE, n fp32, 16-byte aligned; may be the same pointer as base (in-place update).
+ * workspace     as for lc_compress (only the status word is used).
+ * Malformed streams set LC_ERR_FORMAT / LC_ERR_MISMATCH in the status word; `out` is then unspecified
+ * but no out-of-bounds access happens.
+ */
+int lc_recover(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k,
+               uint64_t n, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs);
+
+/* Copies a stream's header to the host. `stream` DEVICE, `info` HOST. Waits for `cs`. */
+int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs);
+
+/* Waits for `cs`, then returns the status word of the last call that used `workspace`. */
+int lc_last_status(const void* workspace, lc_cuda_stream_t cs);
+
+/*
+ * Host-buffer variants: the same two passes for callers whose state lives in host memory (pinned
+ * memory makes the copies asynchronous). Every transfer is part of the call: base, cur -> device,
+ * stream -> host for compress; base, streams -> device, out -> host for recover. The device memory
+ * comes from `arena` (DEVICE, 256-byte aligned, arena_bytes >= lc_host_arena_bytes()); the calls wait
+ * for `cs` before returning and return the device status as well.
+ */
+uint64_t lc_host_arena_bytes(uint64_t n, int nbits, int k);
+
+/* base_host, cur_host HOST fp32[n]; stream_host HOST, capacity >= lc_stream_bound; *stream_bytes_out
+ * receives the stream size. */
+int lc_compress_host(const float* base_host, const float* cur_host, uint64_t n, int nbits,
+                     void* stream_host, uint64_t stream_capacity, uint64_t* stream_bytes_out,
+                     void* arena, uint64_t arena_bytes, lc_cuda_stream_t cs);
+
+/* base_host HOST fp32[n]; streams_host HOST array of k HOST pointers; out_host HOST fp32[n]. */
+int lc_recover_host(const float* base_host, const void* const* streams_host,
+                    const uint64_t* stream_bytes, int k, uint64_t n, float* out_host, void* arena,
+                    uint64_t arena_bytes, lc_cuda_stream_t cs);
+
+/*
+ * Stage dumps for parity tests: results of the statistics and table kernels of the last lc_compress
+ * that used `workspace`. All outputs HOST. Waits for `cs`.
+ *   count[512], mmin[512], mmax[512]: bucket statistics by key = 256*sign + exponent field (empty
+ *   bucket: mmin 0x7FFFFF, mmax 0).
+ *   len[512], code[512]: code length and canonical code of the symbol each key maps to.
+ */
+int lc_debug_bins(const void* workspace, uint64_t* count, uint32_t* mmin, uint32_t* mmax,
+                  lc_cuda_stream_t cs);
+int lc_debug_codes(const void* workspace, uint32_t* len, uint64_t* code, lc_cuda_stream_t cs);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LC_H_ */

@@ -266,6 +266,40 @@ uint64_t element_index(uint64_t c, uint64_t lane, uint64_t j, uint64_t e) {
   return kChunkElems * c + kLanes * kGroup * j + kGroup * lane + e;
 }
 
+// Codes one chunk (format section 2): writes the 32 lane bit counts (u16 each) and the chunk's bytes,
+// returns the chunk's size in bytes (a multiple of 16).
+uint64_t encode_chunk(const float* base, const float* cur, uint64_t n, const Table& t, const Selection& sel,
+                      uint64_t c, uint8_t* lane_index /*[64]*/, uint8_t* chunk, uint64_t* chunk_bits_out) {
+  // first the lane lengths, to know the chunk size, then the bits.
+  uint64_t chunk_bits = 0;
+  for (uint64_t lane = 0; lane < kLanes; ++lane) {
+    uint64_t lane_bits = 0;
+    for (uint64_t j = 0; j < kSteps; ++j)
+      for (uint64_t e = 0; e < kGroup; ++e) {
+        const uint64_t i = element_index(c, lane, j, e);
+        if (i < n) lane_bits += t.len[sel.symbol_of_key[bucket_key(cur[i] - base[i])]];
+      }
+    put_le(lane_index + 2 * lane, lane_bits, 2);
+    chunk_bits += lane_bits;
+  }
+  const uint64_t chunk_bytes = align16((chunk_bits + 7) / 8);
+  std::memset(chunk, 0, chunk_bytes);
+  uint64_t bit = 0;
+  for (uint64_t lane = 0; lane < kLanes; ++lane)
+    for (uint64_t j = 0; j < kSteps; ++j)
+      for (uint64_t e = 0; e < kGroup; ++e) {
+        const uint64_t i = element_index(c, lane, j, e);
+        if (i >= n) continue;
+        const int symbol = sel.symbol_of_key[bucket_key(cur[i] - base[i])];
+        for (int b = t.len[symbol] - 1; b >= 0; --b) {
+          if ((t.code[symbol] >> b) & 1) set_chunk_bit(chunk, bit);
+          bit += 1;
+        }
+      }
+  *chunk_bits_out = chunk_bits;
+  return chunk_bytes;
+}
+
 struct Parsed {
   Table table;
   uint64_t n = 0;
@@ -514,33 +548,9 @@ int lco_compress(const float* base, const float* cur, uint64_t n, int nbits, uin
   uint64_t payload_bits = 0;
   for (uint64_t c = 0; c < L.nchunks; ++c) {
     put_le(chunk_index + 8 * c, payload_bytes, 8);
-    // first the lane lengths, to know the chunk size, then the bits.
     uint64_t chunk_bits = 0;
-    for (uint64_t lane = 0; lane < kLanes; ++lane) {
-      uint64_t lane_bits = 0;
-      for (uint64_t j = 0; j < kSteps; ++j)
-        for (uint64_t e = 0; e < kGroup; ++e) {
-          const uint64_t i = element_index(c, lane, j, e);
-          if (i < n) lane_bits += t.len[sel.symbol_of_key[bucket_key(cur[i] - base[i])]];
-        }
-      put_le(lane_index + 2 * (kLanes * c + lane), lane_bits, 2);
-      chunk_bits += lane_bits;
-    }
-    const uint64_t chunk_bytes = align16((chunk_bits + 7) / 8);
-    uint8_t* chunk = stream + L.payload_off + payload_bytes;
-    std::memset(chunk, 0, chunk_bytes);
-    uint64_t bit = 0;
-    for (uint64_t lane = 0; lane < kLanes; ++lane)
-      for (uint64_t j = 0; j < kSteps; ++j)
-        for (uint64_t e = 0; e < kGroup; ++e) {
-          const uint64_t i = element_index(c, lane, j, e);
-          if (i >= n) continue;
-          const int symbol = sel.symbol_of_key[bucket_key(cur[i] - base[i])];
-          for (int b = t.len[symbol] - 1; b >= 0; --b) {
-            if ((t.code[symbol] >> b) & 1) set_chunk_bit(chunk, bit);
-            bit += 1;
-          }
-        }
+    const uint64_t chunk_bytes = encode_chunk(base, cur, n, t, sel, c, lane_index + 2 * kLanes * c,
+                                              stream + L.payload_off + payload_bytes, &chunk_bits);
     payload_bytes += chunk_bytes;
     payload_bits += chunk_bits;
   }
@@ -604,6 +614,44 @@ int lco_recover(const float* base, const uint8_t* const* streams, const uint64_t
     for (uint64_t i = 0; i < n; ++i) x[i] = x[i] + parsed[j].table.rep[sym[i]];
   }
   for (uint64_t i = 0; i < n; ++i) out[i] = x[i];
+  return LCO_OK;
+}
+
+// Algorithm 1 step 7 computed directly, without a bitstream: out = base + quantized(cur - base).
+int lco_apply_quantized(const float* base, const float* cur, uint64_t n, int nbits, float* out) {
+  if (nbits < 1 || nbits > 8) return LCO_ERR_ARG;
+  std::vector<Bucket> buckets(512);
+  delta_buckets(base, cur, n, buckets.data());
+  Table t;
+  Selection sel;
+  const int rc = build_table(buckets.data(), n, nbits, &t, &sel);
+  if (rc != LCO_OK) return rc;
+  for (uint64_t i = 0; i < n; ++i) out[i] = base[i] + t.rep[sel.symbol_of_key[bucket_key(cur[i] - base[i])]];
+  return LCO_OK;
+}
+
+// Codes only the listed chunks of the stream that lco_compress would write for the whole vector (the
+// table comes from the whole vector). For chunk m: lane_bits[32*m ..] and bytes[m] payload bytes at
+// payload + m*stride. Lets a test check chunks of a vector too large to code in full.
+int lco_compress_chunks(const float* base, const float* cur, uint64_t n, int nbits, const uint64_t* chunk_ids,
+                        uint64_t m, uint16_t* lane_bits, uint8_t* payload, uint64_t stride, uint64_t* bytes) {
+  if (nbits < 1 || nbits > 8) return LCO_ERR_ARG;
+  std::vector<Bucket> buckets(512);
+  delta_buckets(base, cur, n, buckets.data());
+  Table t;
+  Selection sel;
+  const int rc = build_table(buckets.data(), n, nbits, &t, &sel);
+  if (rc != LCO_OK) return rc;
+  std::vector<uint8_t> chunk(kChunkElems * 8 + 16);
+  for (uint64_t k = 0; k < m; ++k) {
+    uint8_t li[64];
+    uint64_t bits = 0;
+    const uint64_t sz = encode_chunk(base, cur, n, t, sel, chunk_ids[k], li, chunk.data(), &bits);
+    if (sz > stride) return LCO_ERR_CAPACITY;
+    for (int lane = 0; lane < 32; ++lane) lane_bits[32 * k + lane] = static_cast<uint16_t>(get_le(li + 2 * lane, 2));
+    std::memcpy(payload + k * stride, chunk.data(), sz);
+    bytes[k] = sz;
+  }
   return LCO_OK;
 }
 

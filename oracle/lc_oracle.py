@@ -33,6 +33,8 @@ def lib():
         L.lco_compress.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_decode_symbols.argtypes = [vp, u64, u64, vp]
         L.lco_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp]
+        L.lco_apply_quantized.argtypes = [vp, vp, u64, i32, vp]
+        L.lco_compress_chunks.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
         _lib = L
     return _lib
 
@@ -142,3 +144,31 @@ def recover(base, streams):
     if rc < 0:
         raise OracleError(rc)
     return out
+
+
+def apply_quantized(base, cur, nbits):
+    """base + quantized(cur - base), computed directly (Algorithm 1 step 7), no bitstream involved."""
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    out = np.zeros(base.size, np.float32)
+    rc = lib().lco_apply_quantized(pb, pc, base.size, nbits, out.ctypes.data)
+    if rc < 0:
+        raise OracleError(rc)
+    return out
+
+
+def compress_chunks(base, cur, nbits, chunk_ids):
+    """(lane_bits[m,32] u16, [payload bytes of each listed chunk]) of the stream for the whole vector."""
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    ids = np.ascontiguousarray(chunk_ids, dtype=np.uint64)
+    m = ids.size
+    stride = 4096 * 8 + 16
+    lane_bits = np.zeros((m, 32), np.uint16)
+    payload = np.zeros(m * stride, np.uint8)
+    sizes = np.zeros(m, np.uint64)
+    rc = lib().lco_compress_chunks(pb, pc, base.size, nbits, ids.ctypes.data, m, lane_bits.ctypes.data,
+                                   payload.ctypes.data, stride, sizes.ctypes.data)
+    if rc < 0:
+        raise OracleError(rc)
+    return lane_bits, [payload[k * stride: k * stride + int(sizes[k])].copy() for k in range(m)]

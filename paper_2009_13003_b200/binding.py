@@ -1,0 +1,204 @@
+"""Thin ctypes binding of ``liblc.so`` (the C ABI in ``include/lc.h``).
+
+Argument marshalling only: every step of the compress and recovery passes runs in the CUDA kernels.
+PyTorch supplies device memory (tensors) and the current CUDA stream. There is no CPU fallback: if the
+library cannot be loaded the import of this module's functions fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+OK, ERR_ARG, ERR_CAPACITY, ERR_NONFINITE, ERR_FORMAT, ERR_MISMATCH, ERR_TIMEOUT, ERR_CUDA = 0, -1, -2, -3, -4, -5, -6, -7
+MAX_CHAIN = 8
+
+SYMBOLS = (
+    "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_recover",
+    "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
+    "lc_debug_bins", "lc_debug_codes",
+)
+
+
+class LCInfo(C.Structure):
+    _fields_ = [
+        ("n", C.c_uint64), ("total_bytes", C.c_uint64), ("payload_bits", C.c_uint64),
+        ("payload_offset", C.c_uint64), ("nbits", C.c_uint32), ("nsym", C.c_uint32),
+        ("max_len", C.c_uint32), ("nchunks", C.c_uint32), ("valid", C.c_int32),
+    ]
+
+
+class LCError(RuntimeError):
+    def __init__(self, code, what=""):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (what, lib().lc_strerror(code).decode(), code))
+
+
+_lib = None
+
+
+def lib():
+    """Loads (building first if the shared object is missing or stale and nvcc is present) liblc.so."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    try:
+        path = _build.build()
+    except Exception as e:  # no nvcc here: use what is in the tree
+        if not os.path.exists(path):
+            raise RuntimeError("liblc.so is missing and could not be built: %s" % e)
+    L = C.CDLL(path)
+    u64, i32, vp = C.c_uint64, C.c_int, C.c_void_p
+    L.lc_version.restype = i32
+    L.lc_strerror.argtypes = [i32]
+    L.lc_strerror.restype = C.c_char_p
+    L.lc_stream_bound.argtypes = [u64, i32]
+    L.lc_stream_bound.restype = u64
+    L.lc_workspace_bytes.argtypes = [u64]
+    L.lc_workspace_bytes.restype = u64
+    L.lc_compress.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp]
+    L.lc_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
+    L.lc_stream_info.argtypes = [vp, C.POINTER(LCInfo), vp]
+    L.lc_last_status.argtypes = [vp, vp]
+    L.lc_host_arena_bytes.argtypes = [u64, i32, i32]
+    L.lc_host_arena_bytes.restype = u64
+    L.lc_compress_host.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), vp, u64, vp]
+    L.lc_recover_host.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
+    L.lc_debug_bins.argtypes = [vp, vp, vp, vp, vp]
+    L.lc_debug_codes.argtypes = [vp, vp, vp]
+    _lib = L
+    return L
+
+
+def _cs(device):
+    return C.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def _check(rc, what):
+    if rc != OK:
+        raise LCError(rc, what)
+
+
+def stream_bound(n: int, nbits: int) -> int:
+    return int(lib().lc_stream_bound(n, nbits))
+
+
+def workspace_bytes(n: int) -> int:
+    return int(lib().lc_workspace_bytes(n))
+
+
+def alloc_workspace(n: int, device) -> torch.Tensor:
+    return torch.empty(workspace_bytes(n), dtype=torch.uint8, device=device)
+
+
+def alloc_stream(n: int, nbits: int, device) -> torch.Tensor:
+    return torch.empty(stream_bound(n, nbits), dtype=torch.uint8, device=device)
+
+
+def _f32_cuda(t, name):
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise ValueError("%s must be a contiguous float32 CUDA tensor" % name)
+    return t
+
+
+def compress_async(base, cur, nbits, stream, workspace):
+    """Enqueues lc_compress on the current stream; no host synchronisation."""
+    _f32_cuda(base, "base"), _f32_cuda(cur, "cur")
+    if base.numel() != cur.numel():
+        raise ValueError("base and cur differ in size")
+    rc = lib().lc_compress(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(),
+                           stream.numel(), workspace.data_ptr(), workspace.numel(), _cs(base.device))
+    _check(rc, "lc_compress")
+
+
+def last_status(workspace) -> int:
+    return int(lib().lc_last_status(workspace.data_ptr(), _cs(workspace.device)))
+
+
+def stream_info(stream) -> LCInfo:
+    info = LCInfo()
+    _check(lib().lc_stream_info(stream.data_ptr(), C.byref(info), _cs(stream.device)), "lc_stream_info")
+    return info
+
+
+def compress(base, cur, nbits, stream=None, workspace=None):
+    """stream <- LC(cur - base). Returns the stream trimmed to its size (a view of ``stream``)."""
+    n = base.numel()
+    if stream is None:
+        stream = alloc_stream(n, nbits, base.device)
+    if workspace is None:
+        workspace = alloc_workspace(n, base.device)
+    compress_async(base, cur, nbits, stream, workspace)
+    _check(last_status(workspace), "lc_compress (device)")
+    info = stream_info(stream)
+    return stream[: info.total_bytes]
+
+
+def recover_async(base, streams, out, workspace):
+    _f32_cuda(base, "base"), _f32_cuda(out, "out")
+    k = len(streams)
+    ptrs = (C.c_void_p * k)(*[s.data_ptr() for s in streams])
+    sizes = (C.c_uint64 * k)(*[s.numel() for s in streams])
+    rc = lib().lc_recover(base.data_ptr(), ptrs, sizes, k, base.numel(), out.data_ptr(), workspace.data_ptr(),
+                          workspace.numel(), _cs(base.device))
+    _check(rc, "lc_recover")
+
+
+def recover(base, streams, out=None, workspace=None):
+    """out <- base + sum of the deltas decoded from ``streams`` (applied in order)."""
+    if out is None:
+        out = torch.empty_like(base)
+    if workspace is None:
+        workspace = alloc_workspace(0, base.device)
+    recover_async(base, streams, out, workspace)
+    _check(last_status(workspace), "lc_recover (device)")
+    return out
+
+
+def host_arena_bytes(n, nbits, k) -> int:
+    return int(lib().lc_host_arena_bytes(n, nbits, k))
+
+
+def compress_host(base_cpu, cur_cpu, nbits, stream_cpu, arena):
+    """Host-buffer compress: copies in, runs, copies the stream out. Returns the stream size."""
+    out = C.c_uint64(0)
+    rc = lib().lc_compress_host(base_cpu.data_ptr(), cur_cpu.data_ptr(), base_cpu.numel(), nbits,
+                                stream_cpu.data_ptr(), stream_cpu.numel(), C.byref(out), arena.data_ptr(),
+                                arena.numel(), _cs(arena.device))
+    _check(rc, "lc_compress_host")
+    return int(out.value)
+
+
+def recover_host(base_cpu, streams_cpu, out_cpu, arena):
+    k = len(streams_cpu)
+    ptrs = (C.c_void_p * k)(*[s.data_ptr() for s in streams_cpu])
+    sizes = (C.c_uint64 * k)(*[s.numel() for s in streams_cpu])
+    rc = lib().lc_recover_host(base_cpu.data_ptr(), ptrs, sizes, k, base_cpu.numel(), out_cpu.data_ptr(),
+                               arena.data_ptr(), arena.numel(), _cs(arena.device))
+    _check(rc, "lc_recover_host")
+    return out_cpu
+
+
+def debug_bins(workspace):
+    import numpy as np
+
+    count = np.zeros(512, np.uint64)
+    mmin = np.zeros(512, np.uint32)
+    mmax = np.zeros(512, np.uint32)
+    _check(lib().lc_debug_bins(workspace.data_ptr(), count.ctypes.data, mmin.ctypes.data, mmax.ctypes.data,
+                               _cs(workspace.device)), "lc_debug_bins")
+    return count, mmin, mmax
+
+
+def debug_codes(workspace):
+    import numpy as np
+
+    ln = np.zeros(512, np.uint32)
+    code = np.zeros(512, np.uint64)
+    _check(lib().lc_debug_codes(workspace.data_ptr(), ln.ctypes.data, code.ctypes.data, _cs(workspace.device)),
+           "lc_debug_codes")
+    return ln, code

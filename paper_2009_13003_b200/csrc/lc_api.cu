@@ -1,0 +1,245 @@
+// C ABI entry points (declared in include/lc.h): argument checks, workspace carving, launch order.
+#include <string.h>
+
+#include "lc_common.cuh"
+
+using namespace lc;
+
+namespace {
+
+bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+struct Carved {
+  Control* ctl;
+  unsigned long long* tiles;
+  uint8_t* eplane;
+  uint32_t* splane;
+};
+
+Carved carve(void* workspace, const WorkspaceLayout& W) {
+  uint8_t* w = static_cast<uint8_t*>(workspace);
+  Carved c;
+  c.ctl = reinterpret_cast<Control*>(w + W.control_off);
+  c.tiles = reinterpret_cast<unsigned long long*>(w + W.tiles_off);
+  c.eplane = w + W.eplane_off;
+  c.splane = reinterpret_cast<uint32_t*>(w + W.splane_off);
+  return c;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lc_version(void) { return 100; }
+
+const char* lc_strerror(int code) {
+  switch (code) {
+    case LC_OK: return "ok";
+    case LC_ERR_ARG: return "invalid argument";
+    case LC_ERR_CAPACITY: return "buffer too small";
+    case LC_ERR_NONFINITE: return "delta contains Inf or NaN";
+    case LC_ERR_FORMAT: return "malformed stream";
+    case LC_ERR_MISMATCH: return "element count mismatch";
+    case LC_ERR_TIMEOUT: return "device-side wait timed out";
+    case LC_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown status";
+  }
+}
+
+uint64_t lc_stream_bound(uint64_t n, int nbits) {
+  if (nbits < 1 || nbits > 8) return 0;
+  const StreamLayout L = stream_layout(n, 1u << nbits);
+  return L.payload_off + (n * (uint64_t)nbits + 7) / 8 + 16 * L.nchunks;
+}
+
+uint64_t lc_workspace_bytes(uint64_t n) { return workspace_layout(n).total; }
+
+int lc_compress(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (!stream || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
+  if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
+    return LC_ERR_ARG;
+  const WorkspaceLayout W = workspace_layout(n);
+  if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
+  const Carved c = carve(workspace, W);
+
+  // control block and tile descriptors start at zero
+  cudaError_t e = cudaMemsetAsync(workspace, 0, W.eplane_off, cs);
+  if (e != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_stats(base, cur, n, c.ctl, c.eplane, c.splane, cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_encode(c.ctl, c.tiles, c.eplane, c.splane, n, static_cast<uint8_t*>(stream), cs)) != cudaSuccess)
+    return LC_ERR_CUDA;
+  return LC_OK;
+}
+
+int lc_recover(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k,
+               uint64_t n, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+  if (k < 1 || k > LC_MAX_CHAIN || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (!streams || !stream_bytes || !workspace || (n > 0 && (!base || !out))) return LC_ERR_ARG;
+  if (!aligned(base, 16) || !aligned(out, 16) || !aligned(workspace, 256)) return LC_ERR_ARG;
+  for (int j = 0; j < k; ++j)
+    if (!streams[j] || !aligned(streams[j], 16)) return LC_ERR_ARG;
+  if (workspace_bytes < sizeof(Control)) return LC_ERR_CAPACITY;
+  Control* ctl = static_cast<Control*>(workspace);
+  cudaError_t e = cudaMemsetAsync(&ctl->status, 0, sizeof(int32_t), cs);
+  if (e != cudaSuccess) return LC_ERR_CUDA;
+  // up to four streams per launch; later launches continue in place from `out`.
+  const float* src = base;
+  for (int first = 0; first < k; first += 4) {
+    const int kk = (k - first) < 4 ? (k - first) : 4;
+    DecodeStreams ds;
+    memset(&ds, 0, sizeof ds);
+    for (int j = 0; j < kk; ++j) {
+      ds.ptr[j] = static_cast<const uint8_t*>(streams[first + j]);
+      ds.bytes[j] = stream_bytes[first + j];
+    }
+    if ((e = launch_decode(src, ds, kk, n, out, &ctl->status, cs)) != cudaSuccess) return LC_ERR_CUDA;
+    src = out;
+  }
+  return LC_OK;
+}
+
+int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
+  if (!stream || !info) return LC_ERR_ARG;
+  uint8_t h[kHeaderBytes];
+  if (cudaMemcpyAsync(h, stream, kHeaderBytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return LC_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return LC_ERR_CUDA;
+  auto le = [&](int off, int bytes) {
+    uint64_t v = 0;
+    for (int b = 0; b < bytes; ++b) v |= (uint64_t)h[off + b] << (8 * b);
+    return v;
+  };
+  memset(info, 0, sizeof *info);
+  info->nbits = h[6];
+  info->n = le(8, 8);
+  info->nsym = (uint32_t)le(16, 4);
+  info->max_len = (uint32_t)le(20, 4);
+  info->nchunks = (uint32_t)le(32, 4);
+  info->payload_bits = le(40, 8);
+  info->total_bytes = le(48, 8);
+  info->payload_offset = le(56, 8);
+  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 &&
+                 le(24, 4) == kChunkElems && le(28, 2) == kLanes && le(30, 2) == kGroup &&
+                 le(36, 4) == kPayloadAlign)
+                    ? 1
+                    : 0;
+  return LC_OK;
+}
+
+int lc_last_status(const void* workspace, lc_cuda_stream_t cs) {
+  if (!workspace) return LC_ERR_ARG;
+  int32_t st = 0;
+  const Control* ctl = static_cast<const Control*>(workspace);
+  if (cudaMemcpyAsync(&st, &ctl->status, sizeof st, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return LC_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return LC_ERR_CUDA;
+  return st;
+}
+
+// ---- host-buffer variants ------------------------------------------------------------------------
+
+uint64_t lc_host_arena_bytes(uint64_t n, int nbits, int k) {
+  if (nbits < 1 || nbits > 8 || k < 1 || k > LC_MAX_CHAIN) return 0;
+  const uint64_t vec = align_up(4 * n, 256);
+  const uint64_t str = align_up(lc_stream_bound(n, nbits), 256);
+  const uint64_t compress = 2 * vec + str;
+  const uint64_t recover = vec + (uint64_t)k * str;
+  return lc_workspace_bytes(n) + (compress > recover ? compress : recover);
+}
+
+int lc_compress_host(const float* base_host, const float* cur_host, uint64_t n, int nbits, void* stream_host,
+                     uint64_t stream_capacity, uint64_t* stream_bytes_out, void* arena, uint64_t arena_bytes,
+                     lc_cuda_stream_t cs) {
+  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (!stream_host || !stream_bytes_out || !arena || !aligned(arena, 256) || (n > 0 && (!base_host || !cur_host)))
+    return LC_ERR_ARG;
+  const uint64_t bound = lc_stream_bound(n, nbits);
+  if (arena_bytes < lc_host_arena_bytes(n, nbits, 1) || stream_capacity < bound) return LC_ERR_CAPACITY;
+  uint8_t* a = static_cast<uint8_t*>(arena);
+  const uint64_t ws_bytes = lc_workspace_bytes(n), vec = align_up(4 * n, 256);
+  float* d_base = reinterpret_cast<float*>(a + ws_bytes);
+  float* d_cur = reinterpret_cast<float*>(a + ws_bytes + vec);
+  uint8_t* d_stream = a + ws_bytes + 2 * vec;
+  if (n > 0) {
+    if (cudaMemcpyAsync(d_base, base_host, 4 * n, cudaMemcpyHostToDevice, cs) != cudaSuccess) return LC_ERR_CUDA;
+    if (cudaMemcpyAsync(d_cur, cur_host, 4 * n, cudaMemcpyHostToDevice, cs) != cudaSuccess) return LC_ERR_CUDA;
+  }
+  int rc = lc_compress(d_base, d_cur, n, nbits, d_stream, bound, a, ws_bytes, cs);
+  if (rc != LC_OK) return rc;
+  if ((rc = lc_last_status(a, cs)) != LC_OK) return rc;
+  lc_info info;
+  if ((rc = lc_stream_info(d_stream, &info, cs)) != LC_OK) return rc;
+  if (!info.valid || info.total_bytes > stream_capacity) return LC_ERR_FORMAT;
+  if (cudaMemcpyAsync(stream_host, d_stream, info.total_bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+    return LC_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return LC_ERR_CUDA;
+  *stream_bytes_out = info.total_bytes;
+  return LC_OK;
+}
+
+int lc_recover_host(const float* base_host, const void* const* streams_host, const uint64_t* stream_bytes, int k,
+                    uint64_t n, float* out_host, void* arena, uint64_t arena_bytes, lc_cuda_stream_t cs) {
+  if (k < 1 || k > LC_MAX_CHAIN || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (!streams_host || !stream_bytes || !arena || !aligned(arena, 256) || (n > 0 && (!base_host || !out_host)))
+    return LC_ERR_ARG;
+  uint8_t* a = static_cast<uint8_t*>(arena);
+  const uint64_t ws_bytes = lc_workspace_bytes(n), vec = align_up(4 * n, 256);
+  uint64_t need = ws_bytes + vec;
+  for (int j = 0; j < k; ++j) {
+    if (!streams_host[j]) return LC_ERR_ARG;
+    need += align_up(stream_bytes[j], 256);
+  }
+  if (arena_bytes < need) return LC_ERR_CAPACITY;
+  float* d_x = reinterpret_cast<float*>(a + ws_bytes);
+  const void* d_streams[LC_MAX_CHAIN];
+  uint64_t off = ws_bytes + vec;
+  if (n > 0 && cudaMemcpyAsync(d_x, base_host, 4 * n, cudaMemcpyHostToDevice, cs) != cudaSuccess) return LC_ERR_CUDA;
+  for (int j = 0; j < k; ++j) {
+    if (cudaMemcpyAsync(a + off, streams_host[j], stream_bytes[j], cudaMemcpyHostToDevice, cs) != cudaSuccess)
+      return LC_ERR_CUDA;
+    d_streams[j] = a + off;
+    off += align_up(stream_bytes[j], 256);
+  }
+  int rc = lc_recover(d_x, d_streams, stream_bytes, k, n, d_x, a, ws_bytes, cs);
+  if (rc != LC_OK) return rc;
+  if ((rc = lc_last_status(a, cs)) != LC_OK) return rc;
+  if (n > 0 && cudaMemcpyAsync(out_host, d_x, 4 * n, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return LC_ERR_CUDA;
+  if (cudaStreamSynchronize(cs) != cudaSuccess) return LC_ERR_CUDA;
+  return LC_OK;
+}
+
+// ---- stage dumps -----------------------------------------------------------------------------------
+
+int lc_debug_bins(const void* workspace, uint64_t* count, uint32_t* mmin, uint32_t* mmax, lc_cuda_stream_t cs) {
+  if (!workspace || !count || !mmin || !mmax) return LC_ERR_ARG;
+  const Control* ctl = static_cast<const Control*>(workspace);
+  static_assert(sizeof(unsigned long long) == sizeof(uint64_t), "");
+  uint32_t inv[kKeys], mx[kKeys];
+  if (cudaMemcpyAsync(count, ctl->count, sizeof ctl->count, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaMemcpyAsync(inv, ctl->inv_min, sizeof inv, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaMemcpyAsync(mx, ctl->max_bits, sizeof mx, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaStreamSynchronize(cs) != cudaSuccess)
+    return LC_ERR_CUDA;
+  for (uint32_t k = 0; k < kKeys; ++k) {
+    mmin[k] = count[k] ? ((~inv[k]) & 0x7FFFFFu) : 0x7FFFFFu;
+    mmax[k] = count[k] ? (mx[k] & 0x7FFFFFu) : 0u;
+  }
+  return LC_OK;
+}
+
+int lc_debug_codes(const void* workspace, uint32_t* len, uint64_t* code, lc_cuda_stream_t cs) {
+  if (!workspace || !len || !code) return LC_ERR_ARG;
+  const Control* ctl = static_cast<const Control*>(workspace);
+  EncEntry enc[kKeys];
+  if (cudaMemcpyAsync(enc, ctl->enc, sizeof enc, cudaMemcpyDeviceToHost, cs) != cudaSuccess ||
+      cudaStreamSynchronize(cs) != cudaSuccess)
+    return LC_ERR_CUDA;
+  for (uint32_t k = 0; k < kKeys; ++k) {
+    len[k] = enc[k].len;
+    code[k] = ((uint64_t)enc[k].code_hi << 32) | enc[k].code_lo;
+  }
+  return LC_OK;
+}
+
+}  // extern "C"

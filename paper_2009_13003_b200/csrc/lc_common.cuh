@@ -1,0 +1,113 @@
+// Shared declarations of the CUDA library: format constants, workspace layout, launcher prototypes.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/lc.h"
+
+namespace lc {
+
+// ---- stream format, version 1 (docs/FORMAT.md) -------------------------------------------------
+constexpr uint32_t kChunkElems = 4096;  // elements per chunk
+constexpr uint32_t kLanes = 32;         // lane sub-streams per chunk (one per warp lane)
+constexpr uint32_t kGroup = 4;          // consecutive elements a lane takes per step (one float4)
+constexpr uint32_t kSteps = kChunkElems / (kLanes * kGroup);  // 32 steps per chunk
+constexpr uint32_t kHeaderBytes = 64;
+constexpr uint32_t kTableEntryBytes = 16;
+constexpr uint32_t kPayloadAlign = 16;
+constexpr uint32_t kKeys = 512;  // 256*sign + exponent field
+
+__host__ __device__ inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+struct StreamLayout {
+  uint64_t nchunks, table_off, chunk_index_off, lane_index_off, payload_off;
+};
+
+__host__ __device__ inline StreamLayout stream_layout(uint64_t n, uint32_t nsym) {
+  StreamLayout L;
+  L.nchunks = (n + kChunkElems - 1) / kChunkElems;
+  L.table_off = kHeaderBytes;
+  L.chunk_index_off = L.table_off + (uint64_t)kTableEntryBytes * nsym;
+  L.lane_index_off = L.chunk_index_off + 8 * (L.nchunks + 1);
+  L.payload_off = align_up(L.lane_index_off + 64 * L.nchunks, kPayloadAlign);
+  return L;
+}
+
+// ---- statistics pass -> encode pass hand-over ("key plane") -----------------------------------
+// The statistics kernel leaves, for every element, its exponent field (1 byte) and its sign (1 bit)
+// in the workspace so that the encode pass reads 1.125 bytes per element instead of 8.
+// A *unit* is 1024 consecutive elements = 8 steps of one chunk, handled by one warp iteration:
+//   exponent plane, unit u: bytes [1024u, 1024u+1024): byte 512*(r/4) + 16*lane + 4*(r%4) + e
+//   sign plane, unit u: u32 word 32u + lane, bit 31 - (4r + e)
+// for step r (0..7) of the unit, lane (0..31) and slot e (0..3), i.e. element 1024u + 128r + 4lane + e.
+constexpr uint32_t kUnitElems = 1024;
+constexpr uint32_t kUnitsPerChunk = kChunkElems / kUnitElems;
+
+// ---- encode pass tiling --------------------------------------------------------------------------
+constexpr uint32_t kEncWarps = 8;  // chunks per tile (one per warp)
+
+// Tile descriptor of the decoupled look-back scan: flag in the top two bits, bytes below.
+constexpr uint64_t kTileFlagShift = 62;
+constexpr uint64_t kTileInvalid = 0, kTileAggregate = 1, kTilePrefix = 2, kTileAbort = 3;
+constexpr uint64_t kTileValueMask = (1ull << kTileFlagShift) - 1;
+
+// Entry of the per-key encode table written by the table kernel.
+struct EncEntry {
+  uint32_t code_lo;  // low 32 bits of the canonical code
+  uint32_t len;      // code length in bits (0..63)
+  uint32_t code_hi;  // bits 32.. of the code (non-zero only when len > 32)
+  uint32_t sym;      // symbol id
+};
+
+// Control block at the start of the workspace. Zeroed at the start of every lc_compress.
+struct Control {
+  int32_t status;         // first device-detected error, 0 if none
+  uint32_t ticket;        // next encode tile
+  uint32_t nsym;          // written by the table kernel
+  uint32_t max_len;       // written by the table kernel
+  uint64_t payload_bits;  // written by the table kernel
+  uint64_t pad_[29];
+  unsigned long long count[kKeys];  // elements per key
+  uint32_t inv_min[kKeys];          // max over the bucket of ~bits (zero-initialised running minimum)
+  uint32_t max_bits[kKeys];         // max over the bucket of bits
+  EncEntry enc[kKeys];
+};
+static_assert(sizeof(Control) % 256 == 0, "control block must keep the planes 256-byte aligned");
+
+struct WorkspaceLayout {
+  uint64_t control_off, tiles_off, eplane_off, splane_off, total;
+  uint64_t ntiles, nunits;
+};
+
+__host__ __device__ inline WorkspaceLayout workspace_layout(uint64_t n) {
+  WorkspaceLayout W;
+  const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
+  W.ntiles = (nchunks + kEncWarps - 1) / kEncWarps;
+  W.nunits = nchunks * kUnitsPerChunk;
+  W.control_off = 0;
+  W.tiles_off = sizeof(Control);
+  W.eplane_off = align_up(W.tiles_off + 8 * W.ntiles, 256);
+  W.splane_off = W.eplane_off + nchunks * kChunkElems;          // 1 byte per element, whole chunks
+  W.total = align_up(W.splane_off + nchunks * (kChunkElems / 8), 256);  // 1 bit per element
+  return W;
+}
+
+// ---- device helpers ----------------------------------------------------------------------------
+__device__ inline void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
+
+// ---- launchers (each defined next to its kernel) ---------------------------------------------------
+cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* eplane,
+                         uint32_t* splane, cudaStream_t cs);
+cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, cudaStream_t cs);
+cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* eplane,
+                          const uint32_t* splane, uint64_t n, uint8_t* stream, cudaStream_t cs);
+
+struct DecodeStreams {
+  const uint8_t* ptr[4];
+  uint64_t bytes[4];
+};
+cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
+                          int32_t* status, cudaStream_t cs);
+
+}  // namespace lc

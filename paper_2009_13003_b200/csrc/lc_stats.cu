@@ -1,0 +1,157 @@
+// Statistics pass: fused delta, (sign, exponent) key extraction, 512-bin histogram with per-bin
+// minimum / maximum, and the 1.125-byte-per-element key plane for the encode pass.
+//
+// Paper: Algorithm 1 step 4 (delta against the tracked state) and Section 3.1.1, exponent-based
+// quantization (bucket = identical sign and exponent; representative from the bucket's min and max).
+//
+// Bound: HBM. 8 bytes per element must be read; 1.125 bytes per element are written.
+//
+// Design for a skewed histogram (a handful of exponents hold almost all elements):
+//  * counts live in shared memory as cnt[key][lane]: every lane of a warp owns its own column, so the
+//    32 atomics of one warp instruction always hit 32 different banks and never the same address,
+//    whatever the keys are;
+//  * min / max are kept per key as a pair of running maxima (of ~bits and of bits: inside one key the
+//    order of the bit patterns is the order of the mantissas). A lane first reads the pair with a
+//    plain load and only issues an atomic when its value would improve it, which after the first few
+//    elements almost never happens;
+//  * counts are integers and min / max are order-free, so the result is deterministic.
+#include "lc_common.cuh"
+
+namespace lc {
+namespace {
+
+constexpr int kStatsThreads = 256;
+constexpr int kRows = 8;  // steps per unit
+constexpr uint32_t kCntWords = kKeys * 32;
+constexpr uint32_t kStatsSmem = (kCntWords + 2 * kKeys) * 4;  // 64 KB + 4 KB
+
+__device__ __forceinline__ float4 ld_stream(const float4* p) {
+  float4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "l"(p));
+  return v;
+}
+
+struct Acc {
+  uint32_t* cnt_lane;  // &cnt[lane]
+  uint2* mm;
+  __device__ __forceinline__ void add(uint32_t bits) {
+    const uint32_t key = bits >> 23;
+    atomicAdd(cnt_lane + key * 32, 1u);
+    const uint2 cur = mm[key];
+    if (~bits > cur.x) atomicMax(&mm[key].x, ~bits);
+    if (bits > cur.y) atomicMax(&mm[key].y, bits);
+  }
+};
+
+__global__ void __launch_bounds__(kStatsThreads, 3)
+stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint64_t n, uint64_t nunits,
+             Control* __restrict__ ctl, uint8_t* __restrict__ eplane, uint32_t* __restrict__ splane) {
+  extern __shared__ __align__(16) uint32_t smem[];
+  uint32_t* cnt = smem;
+  uint2* mm = reinterpret_cast<uint2*>(smem + kCntWords);
+  for (uint32_t i = threadIdx.x; i < kCntWords + 2 * kKeys; i += kStatsThreads) smem[i] = 0;
+  __syncthreads();
+
+  const uint32_t lane = threadIdx.x & 31;
+  const uint64_t warp = (uint64_t)blockIdx.x * (kStatsThreads / 32) + (threadIdx.x >> 5);
+  const uint64_t nwarps = (uint64_t)gridDim.x * (kStatsThreads / 32);
+  Acc acc{cnt + lane, mm};
+
+  for (uint64_t u = warp; u < nunits; u += nwarps) {
+    const uint64_t i0 = u * kUnitElems;
+    uint32_t ew[kRows];
+    uint32_t signs = 0;
+    if (i0 + kUnitElems <= n) {
+      const float4* b4 = reinterpret_cast<const float4*>(base + i0) + lane;
+      const float4* c4 = reinterpret_cast<const float4*>(cur + i0) + lane;
+      float4 b[kRows], c[kRows];
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) {
+        b[r] = ld_stream(b4 + 32 * r);
+        c[r] = ld_stream(c4 + 32 * r);
+      }
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) {
+        const uint32_t d0 = __float_as_uint(__fsub_rn(c[r].x, b[r].x));
+        const uint32_t d1 = __float_as_uint(__fsub_rn(c[r].y, b[r].y));
+        const uint32_t d2 = __float_as_uint(__fsub_rn(c[r].z, b[r].z));
+        const uint32_t d3 = __float_as_uint(__fsub_rn(c[r].w, b[r].w));
+        acc.add(d0);
+        acc.add(d1);
+        acc.add(d2);
+        acc.add(d3);
+        // exponent fields: byte 3 of (bits << 1); gather the four into one word, slot e in byte e.
+        const uint32_t lo = __byte_perm(d0 << 1, d1 << 1, 0x0073);
+        const uint32_t hi = __byte_perm(d2 << 1, d3 << 1, 0x0073);
+        ew[r] = __byte_perm(lo, hi, 0x5410);
+        signs = __funnelshift_l(d0, signs, 1);
+        signs = __funnelshift_l(d1, signs, 1);
+        signs = __funnelshift_l(d2, signs, 1);
+        signs = __funnelshift_l(d3, signs, 1);
+      }
+    } else {
+      // ragged tail: the last units of the vector, element by element.
+#pragma unroll 1
+      for (int r = 0; r < kRows; ++r) {
+        uint32_t word = 0;
+        for (int e = 0; e < 4; ++e) {
+          const uint64_t i = i0 + 128 * r + 4 * lane + e;
+          uint32_t d = 0;
+          if (i < n) {
+            d = __float_as_uint(__fsub_rn(cur[i], base[i]));
+            acc.add(d);
+          }
+          word |= ((d >> 23) & 255u) << (8 * e);
+          signs = __funnelshift_l(d, signs, 1);
+        }
+        ew[r] = word;
+      }
+    }
+    uint4* ep = reinterpret_cast<uint4*>(eplane + i0) + lane;
+    ep[0] = make_uint4(ew[0], ew[1], ew[2], ew[3]);
+    ep[32] = make_uint4(ew[4], ew[5], ew[6], ew[7]);
+    splane[u * 32 + lane] = signs;
+  }
+  __syncthreads();
+
+  // fold the 32 lane columns of each key and merge into the global bins.
+  for (uint32_t key = threadIdx.x; key < kKeys; key += kStatsThreads) {
+    uint32_t total = 0;
+#pragma unroll 8
+    for (uint32_t l = 0; l < 32; ++l) total += cnt[key * 32 + ((l + threadIdx.x) & 31)];
+    if (total != 0) {
+      atomicAdd(&ctl->count[key], (unsigned long long)total);
+      atomicMax(&ctl->inv_min[key], mm[key].x);
+      atomicMax(&ctl->max_bits[key], mm[key].y);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* eplane,
+                         uint32_t* splane, cudaStream_t cs) {
+  const WorkspaceLayout W = workspace_layout(n);
+  if (W.nunits == 0) return cudaSuccess;
+  static int blocks_per_sm = 0, sms = 0;
+  if (blocks_per_sm == 0) {
+    cudaError_t e = cudaFuncSetAttribute(stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmem);
+    if (e != cudaSuccess) return e;
+    int dev = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    int bps = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, stats_kernel, kStatsThreads, kStatsSmem);
+    if (e != cudaSuccess) return e;
+    blocks_per_sm = bps > 0 ? bps : 1;
+  }
+  const uint64_t want = (W.nunits + kStatsThreads / 32 - 1) / (kStatsThreads / 32);
+  const uint64_t full = (uint64_t)sms * blocks_per_sm;
+  const unsigned grid = (unsigned)(want < full ? want : full);
+  stats_kernel<<<grid, kStatsThreads, kStatsSmem, cs>>>(base, cur, n, W.nunits, ctl, eplane, splane);
+  return cudaGetLastError();
+}
+
+}  // namespace lc

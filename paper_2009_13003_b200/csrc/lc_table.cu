@@ -1,0 +1,238 @@
+// Table pass: one CTA turns the 512 bucket statistics into the symbol table of the stream.
+//
+// Paper: Section 3.1.1 (priority promotion: keep the 2^x - 1 occupied buckets with the largest
+// exponent, merge the rest into one bucket of value 0; representative = average of the bucket's
+// minimum and maximum) and Section 3.1.2 (Huffman code over the bucket indices). Tie-breaks and the
+// canonical code assignment are those of the stream format text, sections 1.2-1.4.
+//
+// Latency-only: O(512) work. Writes the stream header and symbol table, and the per-key encode table
+// the encode pass looks codes up in.
+#include "lc_common.cuh"
+
+namespace lc {
+namespace {
+
+constexpr int kTableThreads = 512;
+constexpr int kMaxSym = 256;
+
+__device__ __forceinline__ void store_le(uint8_t* p, uint64_t v, int bytes) {
+  for (int b = 0; b < bytes; ++b) p[b] = (uint8_t)(v >> (8 * b));
+}
+
+__global__ void __launch_bounds__(kTableThreads)
+table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restrict__ stream) {
+  __shared__ uint32_t warp_cand[16];
+  __shared__ uint16_t sym_of_key[kKeys];
+  __shared__ unsigned long long sym_count[kMaxSym];
+  __shared__ uint32_t sym_key[kMaxSym];
+  __shared__ uint32_t sym_rep[kMaxSym];
+  __shared__ uint32_t sym_len[kMaxSym];
+  __shared__ unsigned long long sym_code[kMaxSym];
+  __shared__ unsigned long long node_w[2 * kMaxSym];
+  __shared__ uint16_t node_parent[2 * kMaxSym];
+  __shared__ uint16_t node_depth[2 * kMaxSym];
+  __shared__ uint16_t leaf_sym[kMaxSym];
+  __shared__ uint16_t canon_order[kMaxSym];
+  __shared__ uint32_t s_maxlen;
+  __shared__ unsigned long long s_kept_total, s_payload_bits;
+
+  const int tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
+
+  // ---- non-finite deltas make the vector unencodable ------------------------------------------
+  const bool bad = (tid == 255 || tid == 511) && ctl->count[tid] != 0;
+  if (__syncthreads_or(bad)) {
+    if (tid == 0) {
+      set_status(&ctl->status, LC_ERR_NONFINITE);
+      for (int b = 0; b < 64; ++b) stream[b] = 0;
+    }
+    return;
+  }
+
+  // ---- priority promotion -------------------------------------------------------------------------
+  // thread `tid` < 508 looks at the key of priority position tid: exponent descending, + before -.
+  uint32_t key = 0;
+  unsigned long long cnt = 0;
+  bool cand = false;
+  if (tid < 508) {
+    const uint32_t E = 254 - (tid >> 1), s = tid & 1;
+    key = 256 * s + E;
+    cnt = ctl->count[key];
+    cand = cnt != 0;
+  }
+  if (tid < kMaxSym) {
+    sym_count[tid] = 0;
+    sym_len[tid] = 0;
+    sym_code[tid] = 0;
+    sym_key[tid] = 0;
+    sym_rep[tid] = 0;
+  }
+  sym_of_key[tid] = 0;
+  if (tid == 0) {
+    s_kept_total = 0;
+    s_payload_bits = 0;
+    s_maxlen = 0;
+  }
+  const uint32_t ballot = __ballot_sync(0xffffffffu, cand);
+  if (lane == 0) warp_cand[warp] = __popc(ballot);
+  __syncthreads();
+  uint32_t rank = __popc(ballot & ((1u << lane) - 1));
+  uint32_t ncand = 0;
+  for (int w = 0; w < 16; ++w) {
+    if (w < warp) rank += warp_cand[w];
+    ncand += warp_cand[w];
+  }
+  const uint32_t keep = min((1u << nbits) - 1u, ncand);
+  const uint32_t nsym = keep + 1;
+  if (cand && rank < keep) {
+    const uint32_t sym = rank + 1;
+    sym_of_key[key] = (uint16_t)sym;
+    sym_count[sym] = cnt;
+    sym_key[sym] = key;
+    // midrange of two values with the same sign and exponent, rounded to nearest even, on mantissas.
+    const uint32_t mmin = (~ctl->inv_min[key]) & 0x7FFFFFu;
+    const uint32_t mmax = ctl->max_bits[key] & 0x7FFFFFu;
+    const uint32_t t = mmin + mmax;
+    uint32_t mr = t >> 1;
+    if ((t & 1u) && (mr & 1u)) mr += 1;
+    sym_rep[sym] = (key << 23) | mr;
+    atomicAdd(&s_kept_total, cnt);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    sym_count[0] = n - s_kept_total;
+  }
+  __syncthreads();
+
+  // ---- Huffman lengths: two-queue construction ----------------------------------------------------
+  // queue A = used symbols sorted by (count, id), found with a rank sort.
+  bool used = false;
+  unsigned long long my_count = 0;
+  if (tid < (int)nsym) {
+    my_count = sym_count[tid];
+    used = my_count != 0;
+  }
+  const uint32_t used_ballot = __ballot_sync(0xffffffffu, used);
+  if (lane == 0 && warp < 8) warp_cand[warp] = __popc(used_ballot);
+  __syncthreads();
+  uint32_t nused = 0;
+  for (int w = 0; w < 8; ++w) nused += warp_cand[w];
+  if (used) {
+    uint32_t r = 0;
+    for (uint32_t j = 0; j < nsym; ++j) {
+      const unsigned long long cj = sym_count[j];
+      if (cj != 0 && (cj < my_count || (cj == my_count && (int)j < tid))) r += 1;
+    }
+    node_w[r] = my_count;
+    leaf_sym[r] = (uint16_t)tid;
+  }
+  __syncthreads();
+  if (tid == 0 && nused >= 2) {
+    uint32_t front_a = 0, front_b = nused, next = nused;
+    for (uint32_t merge = 0; merge + 1 < nused; ++merge) {
+      uint32_t pick[2];
+      for (int q = 0; q < 2; ++q) {
+        const bool a_has = front_a < nused, b_has = front_b < next;
+        if (a_has && (!b_has || node_w[front_a] <= node_w[front_b])) pick[q] = front_a++;
+        else pick[q] = front_b++;
+      }
+      node_w[next] = node_w[pick[0]] + node_w[pick[1]];
+      node_parent[pick[0]] = (uint16_t)next;
+      node_parent[pick[1]] = (uint16_t)next;
+      next += 1;
+    }
+    // depths, from the root (the last node) down; parents always have larger indices.
+    const uint32_t root = next - 1;
+    node_depth[root] = 0;
+    for (int v = (int)root - 1; v >= 0; --v) node_depth[v] = node_depth[node_parent[v]] + 1;
+    uint32_t maxlen = 0;
+    unsigned long long bits = 0;
+    for (uint32_t r = 0; r < nused; ++r) {
+      sym_len[leaf_sym[r]] = node_depth[r];
+      maxlen = max(maxlen, (uint32_t)node_depth[r]);
+      bits += node_w[r] * node_depth[r];
+    }
+    s_maxlen = maxlen;
+    s_payload_bits = bits;
+  }
+  __syncthreads();
+
+  // ---- canonical codes: used symbols sorted by (len, id) -------------------------------------------
+  if (used && nused >= 2) {
+    const uint32_t my_len = sym_len[tid];
+    uint32_t r = 0;
+    for (uint32_t j = 0; j < nsym; ++j) {
+      const uint32_t lj = sym_len[j];
+      if (lj != 0 && (lj < my_len || (lj == my_len && (int)j < tid))) r += 1;
+    }
+    canon_order[r] = (uint16_t)tid;
+  }
+  __syncthreads();
+  if (tid == 0 && nused >= 2) {
+    unsigned long long code = 0;
+    uint32_t prev_len = 0;
+    for (uint32_t r = 0; r < nused; ++r) {
+      const uint32_t j = canon_order[r];
+      if (r > 0) code = (code + 1) << (sym_len[j] - prev_len);
+      sym_code[j] = code;
+      prev_len = sym_len[j];
+    }
+  }
+  __syncthreads();
+
+  // ---- outputs ---------------------------------------------------------------------------------------
+  {
+    const uint32_t sym = sym_of_key[tid];
+    EncEntry e;
+    e.code_lo = (uint32_t)sym_code[sym];
+    e.code_hi = (uint32_t)(sym_code[sym] >> 32);
+    e.len = sym_len[sym];
+    e.sym = sym;
+    ctl->enc[tid] = e;
+  }
+  const StreamLayout L = stream_layout(n, nsym);
+  if (tid < (int)nsym) {
+    uint8_t* e = stream + L.table_off + 16 * tid;
+    store_le(e, sym_key[tid], 2);
+    e[2] = (uint8_t)sym_len[tid];
+    e[3] = 0;
+    store_le(e + 4, sym_rep[tid], 4);
+    store_le(e + 8, sym_count[tid], 8);
+  }
+  if (tid == 0) {
+    ctl->nsym = nsym;
+    ctl->max_len = s_maxlen;
+    ctl->payload_bits = s_payload_bits;
+    uint8_t* h = stream;
+    h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
+    store_le(h + 4, 1, 2);
+    h[6] = (uint8_t)nbits;
+    h[7] = 0;
+    store_le(h + 8, n, 8);
+    store_le(h + 16, nsym, 4);
+    store_le(h + 20, s_maxlen, 4);
+    store_le(h + 24, kChunkElems, 4);
+    store_le(h + 28, kLanes, 2);
+    store_le(h + 30, kGroup, 2);
+    store_le(h + 32, L.nchunks, 4);
+    store_le(h + 36, kPayloadAlign, 4);
+    store_le(h + 40, s_payload_bits, 8);
+    store_le(h + 56, L.payload_off, 8);
+    // bytes between the lane index and the payload are zero.
+    for (uint64_t p = L.lane_index_off + 64 * L.nchunks; p < L.payload_off; ++p) stream[p] = 0;
+    if (L.nchunks == 0) {
+      // nothing for the encode pass to do: finish the stream here.
+      store_le(stream + L.chunk_index_off, 0, 8);
+      store_le(h + 48, L.payload_off, 8);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, cudaStream_t cs) {
+  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream);
+  return cudaGetLastError();
+}
+
+}  // namespace lc

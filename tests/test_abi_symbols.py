@@ -1,0 +1,44 @@
+"""The C-ABI library loads without a GPU and exports every function include/lc.h declares."""
+import os
+import re
+
+from conftest import ROOT
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "lc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lc_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2009_13003_b200 import binding
+
+    names = declared_functions()
+    assert "lc_compress" in names and "lc_recover" in names and len(names) >= 10
+    L = binding.lib()
+    for name in names:
+        assert hasattr(L, name), name
+    assert sorted(binding.SYMBOLS) == names
+
+
+def test_host_side_size_functions_match_the_format_text(oracle):
+    from paper_2009_13003_b200 import binding
+
+    for n in (0, 1, 10, 4096, 4097, 61_706, 11_689_512, 1_315_575_808):
+        for nbits in (1, 2, 5, 8):
+            nchunks = (n + 4095) // 4096
+            head = (64 + 16 * 2 ** nbits + 8 * (nchunks + 1) + 64 * nchunks + 15) // 16 * 16
+            want = head + (n * nbits + 7) // 8 + 16 * nchunks
+            assert binding.stream_bound(n, nbits) == want == oracle.stream_bound(n, nbits)
+        assert binding.workspace_bytes(n) >= n + n // 8
+    assert binding.stream_bound(10, 0) == 0 and binding.stream_bound(10, 9) == 0
+
+
+def test_host_argument_checks_need_no_device():
+    from paper_2009_13003_b200 import binding
+
+    L = binding.lib()
+    assert L.lc_compress(None, None, 16, 4, None, 0, None, 0, None) == binding.ERR_ARG
+    assert L.lc_recover(None, None, None, 0, 16, None, None, 0, None) == binding.ERR_ARG
+    assert L.lc_strerror(binding.ERR_FORMAT) == b"malformed stream"
