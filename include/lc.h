@@ -86,6 +86,15 @@ int lc_compress(const float* base, const float* cur, uint64_t n, int nbits, void
                 uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs);
 
 /*
+ * lc_compress with per-kernel timing, for profiling: same arguments and result as lc_compress, but the
+ * call records CUDA events around its three kernels on `cs`, waits for them, and stores the elapsed
+ * milliseconds in kernel_ms (HOST float[3]: statistics pass, table pass, encode pass).
+ */
+int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                      uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs,
+                      float* kernel_ms);
+
+/*
  * Recovery pass (Algorithm 1 step 7 applied k times; u_t = u_0 + sum_i quantized delta_i).
  *   out_i = fl32(...fl32(fl32(base_i + d_0,i) + d_1,i)... + d_{k-1},i), streams applied in array order.
  * base          DEVICE, n fp32, 16-byte aligned.

@@ -17,7 +17,8 @@ OK, ERR_ARG, ERR_CAPACITY, ERR_NONFINITE, ERR_FORMAT, ERR_MISMATCH, ERR_TIMEOUT,
 MAX_CHAIN = 8
 
 SYMBOLS = (
-    "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_recover",
+    "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_timed",
+    "lc_recover",
     "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
     "lc_debug_bins", "lc_debug_codes",
 )
@@ -61,6 +62,7 @@ def lib():
     L.lc_workspace_bytes.argtypes = [u64]
     L.lc_workspace_bytes.restype = u64
     L.lc_compress.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp]
+    L.lc_compress_timed.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, C.POINTER(C.c_float)]
     L.lc_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
     L.lc_stream_info.argtypes = [vp, C.POINTER(LCInfo), vp]
     L.lc_last_status.argtypes = [vp, vp]
@@ -113,6 +115,15 @@ def compress_async(base, cur, nbits, stream, workspace):
     rc = lib().lc_compress(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(),
                            stream.numel(), workspace.data_ptr(), workspace.numel(), _cs(base.device))
     _check(rc, "lc_compress")
+
+
+def compress_timed(base, cur, nbits, stream, workspace):
+    """lc_compress with events around its kernels; returns (stats_ms, table_ms, encode_ms)."""
+    ms = (C.c_float * 3)()
+    rc = lib().lc_compress_timed(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(),
+                                 stream.numel(), workspace.data_ptr(), workspace.numel(), _cs(base.device), ms)
+    _check(rc, "lc_compress_timed")
+    return tuple(float(x) for x in ms)
 
 
 def last_status(workspace) -> int:

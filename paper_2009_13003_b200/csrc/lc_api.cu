@@ -74,6 +74,34 @@ int lc_compress(const float* base, const float* cur, uint64_t n, int nbits, void
   return LC_OK;
 }
 
+int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                      uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs,
+                      float* kernel_ms) {
+  if (!kernel_ms) return LC_ERR_ARG;
+  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (!stream || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
+  if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
+    return LC_ERR_ARG;
+  const WorkspaceLayout W = workspace_layout(n);
+  if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
+  const Carved c = carve(workspace, W);
+  cudaEvent_t ev[4];
+  for (int i = 0; i < 4; ++i)
+    if (cudaEventCreate(&ev[i]) != cudaSuccess) return LC_ERR_CUDA;
+  bool ok = cudaMemsetAsync(workspace, 0, W.eplane_off, cs) == cudaSuccess;
+  ok = ok && cudaEventRecord(ev[0], cs) == cudaSuccess;
+  ok = ok && launch_stats(base, cur, n, c.ctl, c.eplane, c.splane, cs) == cudaSuccess;
+  ok = ok && cudaEventRecord(ev[1], cs) == cudaSuccess;
+  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
+  ok = ok && cudaEventRecord(ev[2], cs) == cudaSuccess;
+  ok = ok && launch_encode(c.ctl, c.tiles, c.eplane, c.splane, n, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
+  ok = ok && cudaEventRecord(ev[3], cs) == cudaSuccess;
+  ok = ok && cudaEventSynchronize(ev[3]) == cudaSuccess;
+  for (int i = 0; ok && i < 3; ++i) ok = cudaEventElapsedTime(&kernel_ms[i], ev[i], ev[i + 1]) == cudaSuccess;
+  for (int i = 0; i < 4; ++i) cudaEventDestroy(ev[i]);
+  return ok ? LC_OK : LC_ERR_CUDA;
+}
+
 int lc_recover(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k,
                uint64_t n, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
   if (k < 1 || k > LC_MAX_CHAIN || n >= (1ull << 32)) return LC_ERR_ARG;
