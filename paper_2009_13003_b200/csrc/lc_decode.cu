@@ -6,9 +6,21 @@
 //
 // One warp decodes one chunk; lane t walks lane sub-stream t of every stream at once, so at step j
 // the warp holds 128 consecutive elements: one coalesced 16-byte load of base and one 16-byte store of
-// out per lane, with the k representatives added in registers in between. Codes are looked up in a
-// shared-memory table indexed by the next kLutBits bits whose entries hold the representative value
-// itself; longer codes take a canonical first-code search.
+// out per lane, with the k representatives added in registers in between.
+//
+//  * The chunk's payload of every stream is first copied, coalesced, into a warp-private staging
+//    area in shared memory; the lanes then pull their words from there. (Reading them straight from
+//    global memory makes every refill touch one cache line per lane.) A chunk that does not fit the
+//    staging area is decoded from global memory by the same code.
+//  * Codes are looked up in shared-memory tables whose entries hold the representative itself. The
+//    first level is indexed by the next kL1Bits bits and replicated 16 times (entry for (index, lane)
+//    at index*16 + lane%16): a 64-bit shared load is served half a warp at a time, so the 16 lanes of
+//    a half-warp always hit 16 different bank pairs although their indices are data dependent.
+//    Longer codes are looked up, by a predicated load, in a plain table on kL2Bits bits and, if longer
+//    still, found by a canonical first-code search.
+//  * A lane keeps a 64-bit bit buffer per stream and tops it up with one predicated word load before
+//    every second symbol; that is enough because two table-resolved codes use at most 2*kL2Bits <= 33
+//    bits.
 //
 // Every read of a stream is bounds-checked against the caller's buffer size and every table is
 // validated before use, so a damaged stream yields LC_ERR_FORMAT (and unspecified output), never an
@@ -21,17 +33,20 @@
 namespace lc {
 namespace {
 
-constexpr int kDecThreads = 256;
-constexpr int kDecWarps = kDecThreads / 32;
-constexpr int kLutBits = 10;
+constexpr int kDecMaxThreads = 512;
+constexpr int kL1Bits = 6;
+constexpr int kL1Rep = 16;
+constexpr int kL2Bits = 10;
 constexpr uint32_t kLongCode = 0xFFFFFFFFu;
+static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill guarantee");
 
-struct StreamState {
-  uint2 lut[1 << kLutBits];          // {bit pattern of rep, code length}; length kLongCode = longer code
-  uint32_t sorted_rep[256];          // representatives in canonical (len, id) order
-  unsigned long long first_code[64]; // first canonical code of each length
-  uint32_t len_count[64];            // codes of each length
-  uint32_t len_offset[64];           // index of the first of them in sorted_rep
+struct alignas(16) StreamState {
+  uint2 l1[(1 << kL1Bits) * kL1Rep];  // {bit pattern of rep, code length}; length kLongCode = not resolved here
+  uint2 l2[1 << kL2Bits];             // same on kL2Bits bits, one copy; length kLongCode = longer code
+  uint32_t sorted_rep[256];           // representatives in canonical (len, id) order
+  unsigned long long first_code[64];  // first canonical code of each length
+  uint32_t len_count[64];             // codes of each length
+  uint32_t len_offset[64];            // index of the first of them in sorted_rep
   // header
   unsigned long long n, payload_bits, total_bytes, payload_off, payload_size;
   unsigned long long chunk_index_off, lane_index_off;
@@ -41,17 +56,30 @@ struct StreamState {
   uint32_t seen_max, nused;
 };
 
+static_assert(sizeof(StreamState) % 16 == 0, "the staging areas behind the tables take 16-byte accesses");
+
 __device__ __forceinline__ uint64_t load_le(const uint8_t* p, int bytes) {
   uint64_t v = 0;
   for (int b = 0; b < bytes; ++b) v |= (uint64_t)p[b] << (8 * b);
   return v;
 }
 
+// Canonical decode of the top `width` bits `idx`: (index into sorted_rep, length) or length 0 if the code
+// is longer than `width`.
+__device__ __forceinline__ uint2 canonical_lookup(const StreamState& S, uint32_t idx, uint32_t width) {
+  for (uint32_t L = 1; L <= width; ++L) {
+    const unsigned long long c = idx >> (width - L);
+    if (c >= S.first_code[L] && c - S.first_code[L] < S.len_count[L])
+      return make_uint2(S.len_offset[L] + (uint32_t)(c - S.first_code[L]), L);
+  }
+  return make_uint2(0u, 0u);
+}
+
 // Parses and validates stream `s`, then builds its decode tables in shared memory. All threads of the
 // CTA call this; returns 0 or the error to report.
 __device__ int prepare_stream(StreamState& S, const uint8_t* __restrict__ s, uint64_t bytes, uint64_t n,
                               int* s_err) {
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, nthreads = blockDim.x;
   if (tid == 0) {
     int err = 0;
     S.kraft = 0; S.count_sum = 0; S.bit_sum = 0; S.seen_max = 0; S.nused = 0; S.only_rep = 0;
@@ -89,7 +117,7 @@ __device__ int prepare_stream(StreamState& S, const uint8_t* __restrict__ s, uin
     }
     *s_err = err;
   }
-  for (int L = tid; L < 64; L += kDecThreads) S.len_count[L] = 0;
+  for (int L = tid; L < 64; L += nthreads) S.len_count[L] = 0;
   __syncthreads();
   if (*s_err) return *s_err;
 
@@ -146,43 +174,76 @@ __device__ int prepare_stream(StreamState& S, const uint8_t* __restrict__ s, uin
     for (int j = 0; j < tid; ++j) r += (s[kHeaderBytes + kTableEntryBytes * j + 2] == my_len) ? 1u : 0u;
     S.sorted_rep[S.len_offset[my_len] + r] = my_rep;
   }
+  if (S.nused < 2 && tid == 0) S.sorted_rep[0] = S.only_rep;
   __syncthreads();
 
-  // ---- lookup table: one thread per entry, canonical decode of the entry's own index
-  for (uint32_t idx = tid; idx < (1u << kLutBits); idx += kDecThreads) {
+  // ---- lookup tables: one thread per entry, canonical decode of the entry's own index
+  for (uint32_t idx = tid; idx < (1u << kL2Bits); idx += nthreads) {
     uint2 ent = make_uint2(0u, kLongCode);
     if (S.nused < 2) {
       ent = make_uint2(S.only_rep, 0u);
     } else {
-      for (uint32_t L = 1; L <= (uint32_t)kLutBits; ++L) {
-        const unsigned long long c = idx >> (kLutBits - L);
-        if (c >= S.first_code[L] && c - S.first_code[L] < S.len_count[L]) {
-          ent = make_uint2(S.sorted_rep[S.len_offset[L] + (uint32_t)(c - S.first_code[L])], L);
-          break;
-        }
-      }
+      const uint2 r = canonical_lookup(S, idx, kL2Bits);
+      if (r.y) ent = make_uint2(S.sorted_rep[r.x], r.y);
     }
-    S.lut[idx] = ent;
+    S.l2[idx] = ent;
+  }
+  for (uint32_t k = tid; k < (1u << kL1Bits) * kL1Rep; k += nthreads) {
+    uint2 ent = make_uint2(0u, kLongCode);
+    if (S.nused < 2) {
+      ent = make_uint2(S.only_rep, 0u);
+    } else {
+      const uint2 r = canonical_lookup(S, k / kL1Rep, kL1Bits);
+      if (r.y) ent = make_uint2(S.sorted_rep[r.x], r.y);
+    }
+    S.l1[k] = ent;
   }
   __syncthreads();
   return 0;
 }
 
-// Bounded word read of a chunk's payload.
-struct ChunkReader {
-  const uint32_t* words;
-  uint32_t nwords;
-  __device__ __forceinline__ uint32_t rd(uint32_t i) const { return i < nwords ? __ldg(words + i) : 0u; }
+// ---- shared-memory access by 32-bit shared address (keeps the hot loop free of generic addressing)
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint2 lds_u64(uint32_t addr) {
+  uint2 v;
+  asm("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// Second-level lookup for the lanes whose first-level entry says "longer code": one predicated load,
+// so that the few lanes that need it do not turn the warp's symbol step into a divergent branch.
+__device__ __forceinline__ void lds_u64_if_long(uint2& ent, uint32_t addr) {
+  asm("{\n\t.reg .pred q;\n\tsetp.gt.u32 q, %1, 63;\n\t@q ld.shared.v2.u32 {%0,%1}, [%2];\n\t}"
+      : "+r"(ent.x), "+r"(ent.y)
+      : "r"(addr));
+}
+
+// Where a chunk's words are read from.
+struct Source {
+  const uint32_t* g;  // chunk words in global memory
+  uint32_t nw;        // words in the chunk
+  uint32_t sbase;     // staged: shared address of the chunk's first word
+  uint32_t slim;      // staged: shared address of the last readable word (zero slack after the chunk)
 };
 
-// Canonical search for a code longer than kLutBits, from bit position p of word wi.
-__device__ __noinline__ uint2 decode_long(const StreamState& S, const uint32_t* words, uint32_t nwords,
-                                          uint32_t wi, uint32_t p, int32_t* status) {
-  const ChunkReader R{words, nwords};
-  const unsigned long long a = ((unsigned long long)R.rd(wi) << 32) | R.rd(wi + 1);
-  const unsigned long long b = R.rd(wi + 2);
+// Canonical search for a code longer than kL2Bits that starts at bit `bitpos` of the chunk.
+__device__ __noinline__ uint2 decode_long(const StreamState& S, const uint32_t* g, uint32_t nw, uint32_t bitpos,
+                                          int32_t* status) {
+  auto rd = [&](uint32_t i) { return i < nw ? __ldg(g + i) : 0u; };
+  const uint32_t wi = bitpos >> 5, p = bitpos & 31;
+  const unsigned long long a = ((unsigned long long)rd(wi) << 32) | rd(wi + 1);
+  const unsigned long long b = rd(wi + 2);
   const unsigned long long window = p ? ((a << p) | (b >> (32 - p))) : a;
-  for (uint32_t L = kLutBits + 1; L <= S.max_len; ++L) {
+  for (uint32_t L = kL2Bits + 1; L <= S.max_len; ++L) {
     const unsigned long long c = window >> (64 - L);
     if (c >= S.first_code[L] && c - S.first_code[L] < S.len_count[L])
       return make_uint2(S.sorted_rep[S.len_offset[L] + (uint32_t)(c - S.first_code[L])], L);
@@ -191,18 +252,160 @@ __device__ __noinline__ uint2 decode_long(const StreamState& S, const uint32_t* 
   return make_uint2(0u, S.max_len ? S.max_len : 1u);
 }
 
-struct LaneCursor {
-  ChunkReader R;
-  uint32_t wi;      // index of w0
-  uint32_t p;       // bit position inside w0
-  uint32_t w0, w1;  // current and next word
+// A lane's read state in one stream of a staged chunk: `cnt` valid bits at the top of hi:lo (the bits
+// below are zero); `next` = shared address of the next word to load.
+struct LaneBits {
+  uint32_t hi, lo;
+  int cnt;
+  uint32_t next;
+
+  __device__ __forceinline__ uint32_t bitpos(const Source& W) const { return (next - W.sbase) * 8u - (uint32_t)cnt; }
+  __device__ __forceinline__ void seek(const Source& W, uint32_t pos) {
+    const uint32_t at = W.sbase + (pos >> 5) * 4u, sh = pos & 31;
+    const uint32_t w0 = lds_u32(min(at, W.slim)), w1 = lds_u32(min(at + 4u, W.slim));
+    hi = __funnelshift_l(w1, w0, sh);
+    lo = w1 << sh;
+    cnt = 64 - (int)sh;
+    next = at + 8u;
+  }
+  // Tops the buffer up with one word if 32 bits or fewer are left; afterwards cnt >= 33. All predicated.
+  __device__ __forceinline__ void refill(uint32_t slim) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred q;\n\t"
+        ".reg .u32 w, t, a;\n\t"
+        "setp.le.s32 q, %2, 32;\n\t"
+        "min.u32 a, %3, %4;\n\t"
+        "@q ld.shared.u32 w, [a];\n\t"
+        "@q shf.r.clamp.b32 t, w, 0, %2;\n\t"   // w >> cnt (0 when cnt == 32)
+        "@q or.b32 %0, %0, t;\n\t"
+        "@q sub.s32 t, 32, %2;\n\t"
+        "@q shf.l.clamp.b32 %1, 0, w, t;\n\t"   // lo was 0: lo = w << (32 - cnt) (0 when cnt == 0)
+        "@q add.s32 %2, %2, 32;\n\t"
+        "@q add.u32 %3, %3, 4;\n\t"
+        "}"
+        : "+r"(hi), "+r"(lo), "+r"(cnt), "+r"(next)
+        : "r"(slim));
+  }
+  __device__ __forceinline__ void consume(uint32_t len) {
+    hi = __funnelshift_l(lo, hi, len);
+    lo <<= len;
+    cnt -= (int)len;
+  }
 };
 
+// Rare path of the staged decoder: this lane met a code longer than kL2Bits. Everything by value, so
+// that the caller's state stays in registers.
+struct LongStep {
+  LaneBits bits;
+  uint32_t rep;
+};
+__device__ __noinline__ LongStep resolve_long(LaneBits B, const StreamState* S, const uint32_t* g, uint32_t nw,
+                                              uint32_t sbase, uint32_t slim, int32_t* status) {
+  Source W{g, nw, sbase, slim};
+  const uint32_t pos = B.bitpos(W);
+  const uint2 ent = decode_long(*S, g, nw, pos, status);
+  B.seek(W, pos + ent.y);
+  return LongStep{B, ent.x};
+}
+
+// Full chunk, every stream staged: the hot loop. Per step a lane decodes 4 elements x KS streams; the
+// KS streams are independent dependency chains and are written interleaved.
 template <int KS>
-__global__ void __launch_bounds__(kDecThreads)
-decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out,
-              int32_t* __restrict__ status) {
-  __shared__ StreamState S[KS];
+__device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const Source* W, const uint32_t* start,
+                                                    const float* base, float* out, uint64_t c, uint32_t lane,
+                                                    int32_t* status) {
+  LaneBits bits[KS];
+  uint32_t l1lane[KS], l2base[KS];
+#pragma unroll
+  for (int s = 0; s < KS; ++s) {
+    bits[s].seek(W[s], start[s]);
+    l1lane[s] = smem_addr(S[s].l1) + (lane & (kL1Rep - 1)) * 8u;
+    l2base[s] = smem_addr(S[s].l2);
+  }
+  const uint64_t e0 = c * kChunkElems + 4 * lane;
+  float4 b = __ldcs(reinterpret_cast<const float4*>(base + e0));
+#pragma unroll 1
+  for (uint32_t j = 0; j < kSteps; ++j) {
+    const uint64_t i = e0 + 128ull * j;
+    float x[4] = {b.x, b.y, b.z, b.w};
+    if (j + 1 < kSteps) b = __ldcs(reinterpret_cast<const float4*>(base + i + 128));
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if ((e & 1) == 0) {
+#pragma unroll
+        for (int s = 0; s < KS; ++s) bits[s].refill(W[s].slim);
+      }
+      uint2 ent[KS];
+#pragma unroll
+      for (int s = 0; s < KS; ++s) ent[s] = lds_u64(l1lane[s] + ((bits[s].hi >> (32 - kL1Bits)) << 7));
+      uint32_t longest = 0;
+#pragma unroll
+      for (int s = 0; s < KS; ++s) {
+        lds_u64_if_long(ent[s], l2base[s] + ((bits[s].hi >> (32 - kL2Bits)) << 3));
+        longest |= ent[s].y;  // lengths are < 64, the marker is all ones
+      }
+      if (__any_sync(0xffffffffu, longest > 63u)) {
+#pragma unroll
+        for (int s = 0; s < KS; ++s) {
+          if (ent[s].y > 63u) {
+            const LongStep r = resolve_long(bits[s], &S[s], W[s].g, W[s].nw, W[s].sbase, W[s].slim, status);
+            bits[s] = r.bits;
+            ent[s] = make_uint2(r.rep, 0u);  // already consumed
+          }
+        }
+      }
+#pragma unroll
+      for (int s = 0; s < KS; ++s) {
+        x[e] = __fadd_rn(x[e], __uint_as_float(ent[s].x));
+        bits[s].consume(ent[s].y);
+      }
+    }
+    __stcs(reinterpret_cast<float4*>(out + i), make_float4(x[0], x[1], x[2], x[3]));
+  }
+}
+static_assert(kL1Rep * 8 == 128, "first-level entries of one index span 128 bytes");
+
+// Any chunk (ragged, or too large to stage), read from global memory; plain code, no warp votes.
+struct GlobalChunk {
+  const uint32_t* g[4];
+  uint32_t nw[4];
+  uint32_t start[4];
+};
+template <int KS>
+__device__ __noinline__ void decode_chunk_global(const StreamState* S, GlobalChunk G, const float* base, float* out,
+                                                 uint64_t c, uint64_t n, uint32_t lane, int32_t* status) {
+  uint32_t pos[KS];
+#pragma unroll
+  for (int s = 0; s < KS; ++s) pos[s] = G.start[s];
+  for (uint32_t j = 0; j < kSteps; ++j) {
+    for (uint32_t e = 0; e < kGroup; ++e) {
+      const uint64_t i = c * kChunkElems + 128ull * j + 4 * lane + e;
+      if (i >= n) continue;
+      float x = base[i];
+#pragma unroll
+      for (int s = 0; s < KS; ++s) {
+        const uint32_t wi = pos[s] >> 5, sh = pos[s] & 31;
+        const uint32_t w0 = wi < G.nw[s] ? __ldg(G.g[s] + wi) : 0u;
+        const uint32_t w1 = wi + 1 < G.nw[s] ? __ldg(G.g[s] + wi + 1) : 0u;
+        const uint32_t peek = __funnelshift_l(w1, w0, sh);
+        uint2 ent = S[s].l2[peek >> (32 - kL2Bits)];
+        if (ent.y > 63u) ent = decode_long(S[s], G.g[s], G.nw[s], pos[s], status);
+        x = __fadd_rn(x, __uint_as_float(ent.x));
+        pos[s] += ent.y;
+      }
+      out[i] = x;
+    }
+  }
+}
+
+// stage_bytes: bytes of staging area per warp and stream (a multiple of 16, at least 32).
+template <int KS>
+__global__ void __launch_bounds__(kDecMaxThreads, 1)
+decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, int32_t* __restrict__ status,
+              uint32_t stage_bytes) {
+  extern __shared__ __align__(16) unsigned char s_raw[];
+  StreamState* S = reinterpret_cast<StreamState*>(s_raw);
   __shared__ int s_err;
 
 #pragma unroll
@@ -214,104 +417,114 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out,
     }
   }
 
-  const uint32_t lane = threadIdx.x & 31;
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
+  unsigned char* stage0 = s_raw + KS * sizeof(StreamState) + (size_t)warp * KS * stage_bytes;
   const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
-  const uint64_t warp0 = (uint64_t)blockIdx.x * kDecWarps + (threadIdx.x >> 5);
-  const uint64_t nwarps = (uint64_t)gridDim.x * kDecWarps;
+  const uint64_t warp0 = (uint64_t)blockIdx.x * warps + warp;
+  const uint64_t nwarps = (uint64_t)gridDim.x * warps;
 
   for (uint64_t c = warp0; c < nchunks; c += nwarps) {
-    LaneCursor cur[KS];
+    Source W[KS];
+    uint32_t start[KS], bytes[KS];
+    unsigned long long off0[KS], off1[KS];
+    bool fits = true;
+    __syncwarp();  // the previous chunk's reads of the staging area are done
+    // all index loads of all streams first, so that their latencies overlap
 #pragma unroll
     for (int s = 0; s < KS; ++s) {
       const uint8_t* sp = streams.ptr[s];
       const unsigned long long* ci = reinterpret_cast<const unsigned long long*>(sp + S[s].chunk_index_off);
-      unsigned long long off0 = __ldg(ci + c), off1 = __ldg(ci + c + 1);
-      if (off0 > off1 || off1 > S[s].payload_size || (off0 & 3) || (off1 & 3)) {
-        set_status(status, LC_ERR_FORMAT);
-        off0 = off1 = 0;
-      }
-      cur[s].R.words = reinterpret_cast<const uint32_t*>(sp + S[s].payload_off + off0);
-      cur[s].R.nwords = (uint32_t)((off1 - off0) >> 2);
+      off0[s] = __ldg(ci + c);
+      off1[s] = __ldg(ci + c + 1);
       const uint16_t* li = reinterpret_cast<const uint16_t*>(sp + S[s].lane_index_off);
-      const uint32_t lane_bits = __ldg(li + c * kLanes + lane);
+      start[s] = __ldg(li + c * kLanes + lane);
+    }
+    // then the asynchronous copies of the payloads into the staging areas
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+      if (off0[s] > off1[s] || off1[s] > S[s].payload_size || (off0[s] & 15) || (off1[s] & 15)) {
+        set_status(status, LC_ERR_FORMAT);
+        off0[s] = off1[s] = 0;
+      }
+      bytes[s] = (uint32_t)min(off1[s] - off0[s], (unsigned long long)kChunkElems * 8);
+      const uint8_t* g = streams.ptr[s] + S[s].payload_off + off0[s];
+      unsigned char* st = stage0 + (size_t)s * stage_bytes;
+      W[s].g = reinterpret_cast<const uint32_t*>(g);
+      W[s].nw = bytes[s] >> 2;
+      W[s].sbase = smem_addr(st);
+      W[s].slim = W[s].sbase + bytes[s] + 12;
+      // 16 bytes of zero slack after the chunk must fit too
+      if (bytes[s] + 16 <= stage_bytes) {
+        for (uint32_t k = lane * 16; k < bytes[s]; k += 32 * 16) cp_async_16(W[s].sbase + k, g + k);
+        if (lane == 0) *reinterpret_cast<uint4*>(st + bytes[s]) = make_uint4(0, 0, 0, 0);
+      } else {
+        fits = false;
+      }
+    }
+    cp_async_commit();
+    // lane start offsets (exclusive scan of the lane bit counts) while the copies are in flight
+#pragma unroll
+    for (int s = 0; s < KS; ++s) {
+      const uint32_t lane_bits = start[s];
       uint32_t incl = lane_bits;
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) {
         const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
         if ((int)lane >= d) incl += v;
       }
-      const uint32_t start = incl - lane_bits;
-      cur[s].wi = start >> 5;
-      cur[s].p = start & 31;
-      cur[s].w0 = cur[s].R.rd(cur[s].wi);
-      cur[s].w1 = cur[s].R.rd(cur[s].wi + 1);
+      start[s] = min(incl - lane_bits, bytes[s] * 8u);
     }
-
-    const uint64_t e0 = c * kChunkElems + 4 * lane;
-    const bool full = (c + 1) * kChunkElems <= n;
-    for (uint32_t j = 0; j < kSteps; ++j) {
-      const uint64_t i = e0 + 128ull * j;
-      float x[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t nvalid = 4;
-      if (full) {
-        const float4 b = __ldcs(reinterpret_cast<const float4*>(base + i));
-        x[0] = b.x; x[1] = b.y; x[2] = b.z; x[3] = b.w;
-      } else {
-        nvalid = i >= n ? 0u : (uint32_t)min((unsigned long long)4, (unsigned long long)(n - i));
+    cp_async_wait_all();
+    __syncwarp();
+    if (fits && (c + 1) * kChunkElems <= n) decode_chunk_staged<KS>(S, W, start, base, out, c, lane, status);
+    else {
+      GlobalChunk G;
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if ((uint32_t)e < nvalid) x[e] = base[i + e];
+      for (int s = 0; s < KS; ++s) {
+        G.g[s] = W[s].g;
+        G.nw[s] = W[s].nw;
+        G.start[s] = start[s];
       }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (!full && (uint32_t)e >= nvalid) break;
-#pragma unroll
-        for (int s = 0; s < KS; ++s) {
-          LaneCursor& C = cur[s];
-          const uint32_t peek = __funnelshift_l(C.w1, C.w0, C.p);
-          uint2 ent = S[s].lut[peek >> (32 - kLutBits)];
-          if (ent.y == kLongCode) ent = decode_long(S[s], C.R.words, C.R.nwords, C.wi, C.p, status);
-          x[e] = __fadd_rn(x[e], __uint_as_float(ent.x));
-          C.p += ent.y;
-          while (C.p >= 32) {
-            C.p -= 32;
-            C.wi += 1;
-            C.w0 = C.w1;
-            C.w1 = C.R.rd(C.wi + 1);
-          }
-        }
-      }
-      if (full) {
-        __stcs(reinterpret_cast<float4*>(out + i), make_float4(x[0], x[1], x[2], x[3]));
-      } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if ((uint32_t)e < nvalid) out[i + e] = x[e];
-      }
+      decode_chunk_global<KS>(S, G, base, out, c, n, lane, status);
     }
   }
 }
 
+constexpr uint32_t kSmemPerSm = 227 * 1024;  // usable shared memory of one CTA on sm_100
+
 template <int KS>
 cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, uint64_t n, float* out,
                              int32_t* status, cudaStream_t cs) {
-  static int blocks_per_sm = 0, sms = 0;
-  if (blocks_per_sm == 0) {
-    int dev = 0;
+  static int sms = 0;
+  constexpr uint32_t kTables = KS * sizeof(StreamState);
+  constexpr uint32_t kMaxDyn = kSmemPerSm - 1024;  // leave room for the static __shared__ variables
+  if (sms == 0) {
+    int dev = 0, v = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    int bps = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, decode_kernel<KS>, kDecThreads, 0);
+    if ((e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDyn);
     if (e != cudaSuccess) return e;
-    blocks_per_sm = bps > 0 ? bps : 1;
+    sms = v;
   }
   const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
-  uint64_t want = (nchunks + kDecWarps - 1) / kDecWarps;
+  // One CTA per SM. Staging per warp and stream: 1.06 x the largest average chunk of the streams (from
+  // the buffer sizes, which bound the payload), with as many warps (16, 12 or 8) as then fit.
+  uint64_t avg = 0;
+  for (int s = 0; s < KS; ++s) {
+    const uint64_t a = streams.bytes[s] / (nchunks ? nchunks : 1);
+    avg = a > avg ? a : avg;
+  }
+  const uint64_t want_stage = align_up(avg + avg / 16 + 64, 16);
+  uint32_t warps = 16;
+  while (warps > 8 && kTables + (uint64_t)warps * KS * want_stage > kMaxDyn) warps -= 4;
+  uint32_t stage = ((kMaxDyn - kTables) / (warps * KS)) / 16 * 16;
+  if (stage > kChunkElems * 8 + 16) stage = kChunkElems * 8 + 16;
+  const uint32_t dyn = kTables + warps * KS * stage;
+  uint64_t want = (nchunks + warps - 1) / warps;
   if (want == 0) want = 1;  // still validates the streams
-  const uint64_t full = (uint64_t)sms * blocks_per_sm;
-  const unsigned grid = (unsigned)(want < full ? want : full);
-  decode_kernel<KS><<<grid, kDecThreads, 0, cs>>>(base, streams, n, out, status);
+  const unsigned grid = (unsigned)(want < (uint64_t)sms ? want : (uint64_t)sms);
+  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, stage);
   return cudaGetLastError();
 }
 
