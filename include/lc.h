@@ -147,6 +147,31 @@ int lc_debug_bins(const void* workspace, uint64_t* count, uint32_t* mmin, uint32
                   lc_cuda_stream_t cs);
 int lc_debug_codes(const void* workspace, uint32_t* len, uint64_t* code, lc_cuda_stream_t cs);
 
+/*
+ * Compress pass without a caller-supplied workspace. (No counterpart in the paper: this is a
+ * deployment variant of lc_compress.)
+ *
+ * For callers that must not allocate device memory when they take a snapshot: a trainer whose
+ * memory pool already owns the whole device, code inside a region where cudaMalloc is forbidden or
+ * would stall the device, a plug-in that is handed raw pointers only. The scratch memory that
+ * lc_compress takes from its caller is here a fixed array inside the library image, so the call
+ * allocates nothing (no cudaMalloc, cudaFree or allocating library routine) and serves vectors of at
+ * most LC_NOALLOC_MAX_N elements; a larger n returns LC_ERR_CAPACITY.
+ *
+ *  - base, cur, n, nbits, stream, stream_capacity: exactly as for lc_compress (DEVICE pointers,
+ *    16-byte aligned); the stream written is byte-identical to lc_compress's.
+ *  - The call waits for `cs` and returns the device status as well (LC_ERR_NONFINITE, LC_ERR_TIMEOUT).
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current). Make that first call outside any CUDA stream capture.
+ *  - Every call on a device shares the one array, which keeps the previous call's contents (the call
+ *    clears what must start at zero). Two calls that overlap on the same GPU race: do not issue them
+ *    from different streams or threads at the same time.
+ *  - The array (about 4.8 MB) stays resident on every GPU that loads the library, until exit.
+ */
+#define LC_NOALLOC_MAX_N 4194304ull
+int lc_compress_noalloc(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                        uint64_t stream_capacity, lc_cuda_stream_t cs);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,8 +20,9 @@ SYMBOLS = (
     "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_timed",
     "lc_recover",
     "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
-    "lc_debug_bins", "lc_debug_codes",
+    "lc_debug_bins", "lc_debug_codes", "lc_compress_noalloc",
 )
+NOALLOC_MAX_N = 4194304
 
 
 class LCInfo(C.Structure):
@@ -70,6 +71,7 @@ def lib():
     L.lc_host_arena_bytes.restype = u64
     L.lc_compress_host.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), vp, u64, vp]
     L.lc_recover_host.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
+    L.lc_compress_noalloc.argtypes = [vp, vp, u64, i32, vp, u64, vp]
     L.lc_debug_bins.argtypes = [vp, vp, vp, vp, vp]
     L.lc_debug_codes.argtypes = [vp, vp, vp]
     _lib = L
@@ -213,3 +215,16 @@ def debug_codes(workspace):
     _check(lib().lc_debug_codes(workspace.data_ptr(), ln.ctypes.data, code.ctypes.data, _cs(workspace.device)),
            "lc_debug_codes")
     return ln, code
+
+
+def compress_noalloc(base, cur, nbits, stream):
+    """lc_compress_noalloc: compress with the library's built-in scratch (n <= NOALLOC_MAX_N).
+
+    For callers that cannot allocate device memory when a snapshot is taken. Waits for the current
+    stream; returns the stream trimmed to its size. Calls must not overlap on one GPU.
+    """
+    _f32_cuda(base, "base"), _f32_cuda(cur, "cur")
+    rc = lib().lc_compress_noalloc(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(),
+                                   stream.numel(), _cs(base.device))
+    _check(rc, "lc_compress_noalloc")
+    return stream[: stream_info(stream).total_bytes]
