@@ -40,11 +40,22 @@ constexpr int kL2Bits = 10;
 constexpr uint32_t kLongCode = 0xFFFFFFFFu;
 static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill guarantee");
 
+// The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory, so that an
+// entry's address is (table base | index bits), one logic operation, with both index fields taken from
+// the same shifted copy of the bit buffer.
+constexpr uint32_t kTableBytes = 8192;
+static_assert((1 << kL1Bits) * kL1Rep * 8 == kTableBytes && (8 << kL2Bits) == kTableBytes, "table sizes");
+constexpr uint32_t kL1Mask = ((1u << kL1Bits) - 1) << 7;  // index * 128 bytes (16 copies of 8 bytes)
+constexpr uint32_t kL2Mask = ((1u << kL2Bits) - 1) << 3;  // index * 8 bytes
+constexpr int kIndexShift = 19;                           // (hi >> 19) & mask == index << (7 or 3)
+static_assert(32 - kL1Bits - 7 == kIndexShift && 32 - kL2Bits - 3 == kIndexShift, "index fields must align");
+
 struct alignas(16) StreamState {
-  uint2 l1[(1 << kL1Bits) * kL1Rep];  // {bit pattern of rep, code length}; length kLongCode = not resolved here
-  uint2 l2[1 << kL2Bits];             // same on kL2Bits bits, one copy; length kLongCode = longer code
+  uint2* l1;  // [(1 << kL1Bits) * kL1Rep] {bit pattern of rep, code length}; length kLongCode = not resolved here
+  uint2* l2;  // [1 << kL2Bits] same on kL2Bits bits, one copy; length kLongCode = longer code
   uint32_t sorted_rep[256];           // representatives in canonical (len, id) order
   unsigned long long first_code[64];  // first canonical code of each length
+  unsigned long long last_aligned[64]; // largest left-aligned 64-bit window whose code has at most this length
   uint32_t len_count[64];             // codes of each length
   uint32_t len_offset[64];            // index of the first of them in sorted_rep
   // header
@@ -77,11 +88,13 @@ __device__ __forceinline__ uint2 canonical_lookup(const StreamState& S, uint32_t
 
 // Parses and validates stream `s`, then builds its decode tables in shared memory. All threads of the
 // CTA call this; returns 0 or the error to report.
-__device__ int prepare_stream(StreamState& S, const uint8_t* __restrict__ s, uint64_t bytes, uint64_t n,
-                              int* s_err) {
+__device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8_t* __restrict__ s,
+                              uint64_t bytes, uint64_t n, int* s_err) {
   const int tid = threadIdx.x, nthreads = blockDim.x;
   if (tid == 0) {
     int err = 0;
+    S.l1 = reinterpret_cast<uint2*>(tables);
+    S.l2 = reinterpret_cast<uint2*>(tables + kTableBytes);
     S.kraft = 0; S.count_sum = 0; S.bit_sum = 0; S.seen_max = 0; S.nused = 0; S.only_rep = 0;
     if (bytes < kHeaderBytes) {
       err = LC_ERR_FORMAT;
@@ -164,6 +177,11 @@ __device__ int prepare_stream(StreamState& S, const uint8_t* __restrict__ s, uin
     }
     S.first_code[0] = 0;
     S.len_offset[0] = 0;
+    // codes of length <= L fill the left-aligned range [0, (first_code[L] + count[L]) << (64 - L))
+    for (int L = 1; L < 64; ++L) {
+      const unsigned long long end = (S.first_code[L] + S.len_count[L]) << (64 - L);  // 0 when the range is everything
+      S.last_aligned[L] = end - 1;
+    }
     *s_err = err;
   }
   __syncthreads();
@@ -212,6 +230,12 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
 __device__ __forceinline__ uint2 lds_u64(uint32_t addr) {
   uint2 v;
   asm("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
+// Streaming 16-byte load; volatile so that it stays where it is written (early in the loop body).
+__device__ __forceinline__ float4 ldg_stream_v4(const float* p) {
+  float4 v;
+  asm volatile("ld.global.cs.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
   return v;
 }
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
@@ -294,19 +318,26 @@ struct LaneBits {
   }
 };
 
-// Rare path of the staged decoder: this lane met a code longer than kL2Bits. Everything by value, so
-// that the caller's state stays in registers.
-struct LongStep {
-  LaneBits bits;
-  uint32_t rep;
-};
-__device__ __noinline__ LongStep resolve_long(LaneBits B, const StreamState* S, const uint32_t* g, uint32_t nw,
-                                              uint32_t sbase, uint32_t slim, int32_t* status) {
-  Source W{g, nw, sbase, slim};
+// Code longer than kL2Bits in a staged chunk: canonical search on a 64-bit window read from the
+// staging area, then re-seat the lane's bit buffer behind the code. Returns the representative.
+__device__ __forceinline__ uint32_t long_code_staged(LaneBits& B, const StreamState& S, const Source& W,
+                                                     int32_t* status) {
   const uint32_t pos = B.bitpos(W);
-  const uint2 ent = decode_long(*S, g, nw, pos, status);
-  B.seek(W, pos + ent.y);
-  return LongStep{B, ent.x};
+  const uint32_t at = W.sbase + (pos >> 5) * 4u, sh = pos & 31;
+  const uint32_t w0 = lds_u32(min(at, W.slim)), w1 = lds_u32(min(at + 4u, W.slim)), w2 = lds_u32(min(at + 8u, W.slim));
+  const unsigned long long window =
+      ((unsigned long long)__funnelshift_l(w1, w0, sh) << 32) | __funnelshift_l(w2, w1, sh);
+  uint32_t L = kL2Bits + 1;
+  while (L < S.max_len && window > S.last_aligned[L]) L += 1;
+  const unsigned long long code = window >> (64 - L);
+  uint32_t rep = 0;
+  if (L <= S.max_len && code >= S.first_code[L] && code - S.first_code[L] < S.len_count[L]) {
+    rep = S.sorted_rep[S.len_offset[L] + (uint32_t)(code - S.first_code[L])];
+  } else {
+    set_status(status, LC_ERR_FORMAT);  // no code matches: damaged payload
+  }
+  B.seek(W, pos + L);
+  return rep;
 }
 
 // Full chunk, every stream staged: the hot loop. Per step a lane decodes 4 elements x KS streams; the
@@ -320,16 +351,17 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
     bits[s].seek(W[s], start[s]);
-    l1lane[s] = smem_addr(S[s].l1) + (lane & (kL1Rep - 1)) * 8u;
+    l1lane[s] = smem_addr(S[s].l1) | ((lane & (kL1Rep - 1)) * 8u);
     l2base[s] = smem_addr(S[s].l2);
   }
   const uint64_t e0 = c * kChunkElems + 4 * lane;
-  float4 b = __ldcs(reinterpret_cast<const float4*>(base + e0));
+  float4 b = ldg_stream_v4(base + e0);
 #pragma unroll 1
   for (uint32_t j = 0; j < kSteps; ++j) {
     const uint64_t i = e0 + 128ull * j;
     float x[4] = {b.x, b.y, b.z, b.w};
-    if (j + 1 < kSteps) b = __ldcs(reinterpret_cast<const float4*>(base + i + 128));
+    // next step's 16 bytes of base, requested a whole step ahead (the last step re-reads its own)
+    b = ldg_stream_v4(base + i + (j + 1 < kSteps ? 128 : 0));
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       if ((e & 1) == 0) {
@@ -338,21 +370,17 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
       }
       uint2 ent[KS];
 #pragma unroll
-      for (int s = 0; s < KS; ++s) ent[s] = lds_u64(l1lane[s] + ((bits[s].hi >> (32 - kL1Bits)) << 7));
+      for (int s = 0; s < KS; ++s) ent[s] = lds_u64(l1lane[s] | ((bits[s].hi >> kIndexShift) & kL1Mask));
       uint32_t longest = 0;
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        lds_u64_if_long(ent[s], l2base[s] + ((bits[s].hi >> (32 - kL2Bits)) << 3));
+        lds_u64_if_long(ent[s], l2base[s] | ((bits[s].hi >> kIndexShift) & kL2Mask));
         longest |= ent[s].y;  // lengths are < 64, the marker is all ones
       }
       if (__any_sync(0xffffffffu, longest > 63u)) {
 #pragma unroll
         for (int s = 0; s < KS; ++s) {
-          if (ent[s].y > 63u) {
-            const LongStep r = resolve_long(bits[s], &S[s], W[s].g, W[s].nw, W[s].sbase, W[s].slim, status);
-            bits[s] = r.bits;
-            ent[s] = make_uint2(r.rep, 0u);  // already consumed
-          }
+          if (ent[s].y > 63u) ent[s] = make_uint2(long_code_staged(bits[s], S[s], W[s], status), 0u);  // consumed
         }
       }
 #pragma unroll
@@ -404,13 +432,15 @@ template <int KS>
 __global__ void __launch_bounds__(kDecMaxThreads, 1)
 decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, int32_t* __restrict__ status,
               uint32_t stage_bytes) {
+  // dynamic shared memory: [pad to 8 KB | 2 tables per stream | StreamState per stream | staging areas]
   extern __shared__ __align__(16) unsigned char s_raw[];
-  StreamState* S = reinterpret_cast<StreamState*>(s_raw);
+  unsigned char* tables = s_raw + ((kTableBytes - (smem_addr(s_raw) & (kTableBytes - 1))) & (kTableBytes - 1));
+  StreamState* S = reinterpret_cast<StreamState*>(s_raw + kTableBytes + KS * 2 * kTableBytes);
   __shared__ int s_err;
 
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
-    const int err = prepare_stream(S[s], streams.ptr[s], streams.bytes[s], n, &s_err);
+    const int err = prepare_stream(S[s], tables + s * 2 * kTableBytes, streams.ptr[s], streams.bytes[s], n, &s_err);
     if (err) {
       if (threadIdx.x == 0) set_status(status, err);
       return;
@@ -418,7 +448,7 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
   }
 
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
-  unsigned char* stage0 = s_raw + KS * sizeof(StreamState) + (size_t)warp * KS * stage_bytes;
+  unsigned char* stage0 = reinterpret_cast<unsigned char*>(S + KS) + (size_t)warp * KS * stage_bytes;
   const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
   const uint64_t warp0 = (uint64_t)blockIdx.x * warps + warp;
   const uint64_t nwarps = (uint64_t)gridDim.x * warps;
@@ -496,7 +526,7 @@ template <int KS>
 cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, uint64_t n, float* out,
                              int32_t* status, cudaStream_t cs) {
   static int sms = 0;
-  constexpr uint32_t kTables = KS * sizeof(StreamState);
+  constexpr uint32_t kTables = kTableBytes + KS * (2 * kTableBytes + sizeof(StreamState));
   constexpr uint32_t kMaxDyn = kSmemPerSm - 1024;  // leave room for the static __shared__ variables
   if (sms == 0) {
     int dev = 0, v = 0;
@@ -508,14 +538,15 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
     sms = v;
   }
   const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
-  // One CTA per SM. Staging per warp and stream: 1.06 x the largest average chunk of the streams (from
+  // One CTA per SM. Staging per warp and stream: 1.03 x the largest average chunk of the streams (from
   // the buffer sizes, which bound the payload), with as many warps (16, 12 or 8) as then fit.
   uint64_t avg = 0;
   for (int s = 0; s < KS; ++s) {
-    const uint64_t a = streams.bytes[s] / (nchunks ? nchunks : 1);
+    const uint64_t index_bytes = 72 * nchunks;  // lane and chunk index entries are not staged
+    const uint64_t a = (streams.bytes[s] > index_bytes ? streams.bytes[s] - index_bytes : 0) / (nchunks ? nchunks : 1);
     avg = a > avg ? a : avg;
   }
-  const uint64_t want_stage = align_up(avg + avg / 16 + 64, 16);
+  const uint64_t want_stage = align_up(avg + avg / 32 + 48, 16);
   uint32_t warps = 16;
   while (warps > 8 && kTables + (uint64_t)warps * KS * want_stage > kMaxDyn) warps -= 4;
   uint32_t stage = ((kMaxDyn - kTables) / (warps * KS)) / 16 * 16;
