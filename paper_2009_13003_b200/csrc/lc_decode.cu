@@ -16,10 +16,11 @@
 //    first level is indexed by the next kL1Bits bits and replicated 16 times (entry for (index, lane)
 //    at index*16 + lane%16): a 64-bit shared load is served half a warp at a time, so the 16 lanes of
 //    a half-warp always hit 16 different bank pairs although their indices are data dependent.
-//    Longer codes are looked up, by a predicated load, in a plain table on kL2Bits bits and, if longer
-//    still, found by a canonical first-code search.
+//    An entry whose 6-bit prefix belongs to longer codes points to a 64-entry sub-table indexed by the
+//    next 6 bits (one predicated load, no branch), which resolves codes of up to 12 bits; still longer
+//    codes are found by a canonical search behind a warp vote.
 //  * A lane keeps a 64-bit bit buffer per stream and tops it up with one predicated word load before
-//    every second symbol; that is enough because two table-resolved codes use at most 2*kL2Bits <= 33
+//    every second symbol; that is enough because two table-resolved codes use at most 2*12 <= 33
 //    bits.
 //
 // Every read of a stream is bounds-checked against the caller's buffer size and every table is
@@ -36,7 +37,10 @@ namespace {
 constexpr int kDecMaxThreads = 512;
 constexpr int kL1Bits = 6;
 constexpr int kL1Rep = 16;
-constexpr int kL2Bits = 10;
+constexpr int kSubBits = 6;                        // second level: the next 6 bits
+constexpr int kL2Bits = kL1Bits + kSubBits;        // longest code the two table levels resolve
+constexpr int kSubTables = 16;                     // 15 usable + one that only says "longer"
+constexpr uint32_t kSubBytes = (1u << kSubBits) * 8;
 constexpr uint32_t kLongCode = 0xFFFFFFFFu;
 static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill guarantee");
 
@@ -44,15 +48,15 @@ static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill g
 // entry's address is (table base | index bits), one logic operation, with both index fields taken from
 // the same shifted copy of the bit buffer.
 constexpr uint32_t kTableBytes = 8192;
-static_assert((1 << kL1Bits) * kL1Rep * 8 == kTableBytes && (8 << kL2Bits) == kTableBytes, "table sizes");
-constexpr uint32_t kL1Mask = ((1u << kL1Bits) - 1) << 7;  // index * 128 bytes (16 copies of 8 bytes)
-constexpr uint32_t kL2Mask = ((1u << kL2Bits) - 1) << 3;  // index * 8 bytes
-constexpr int kIndexShift = 19;                           // (hi >> 19) & mask == index << (7 or 3)
-static_assert(32 - kL1Bits - 7 == kIndexShift && 32 - kL2Bits - 3 == kIndexShift, "index fields must align");
+static_assert((1 << kL1Bits) * kL1Rep * 8 == kTableBytes && kSubTables * kSubBytes == kTableBytes, "table sizes");
+constexpr uint32_t kL1Mask = ((1u << kL1Bits) - 1) << 7;    // index * 128 bytes (16 copies of 8 bytes)
+constexpr int kL1Shift = 32 - kL1Bits - 7;                  // (hi >> 19) & kL1Mask == first-level index * 128
+constexpr uint32_t kSubMask = ((1u << kSubBits) - 1) << 3;  // index * 8 bytes
+constexpr int kSubShift = 32 - kL1Bits - kSubBits - 3;      // (hi >> 17) & kSubMask == sub-table index * 8
 
 struct alignas(16) StreamState {
   uint2* l1;  // [(1 << kL1Bits) * kL1Rep] {bit pattern of rep, code length}; length kLongCode = not resolved here
-  uint2* l2;  // [1 << kL2Bits] same on kL2Bits bits, one copy; length kLongCode = longer code
+  uint2* sub; // [kSubTables][1 << kSubBits] second level: {rep, length} or length kLongCode = longer code
   uint32_t sorted_rep[256];           // representatives in canonical (len, id) order
   unsigned long long first_code[64];  // first canonical code of each length
   unsigned long long last_aligned[64]; // largest left-aligned 64-bit window whose code has at most this length
@@ -64,10 +68,13 @@ struct alignas(16) StreamState {
   uint32_t nsym, max_len, nchunks, only_rep;
   // validation accumulators
   unsigned long long kraft, count_sum, bit_sum;
-  uint32_t seen_max, nused;
+  uint32_t seen_max, nused, nsub;
+  uint8_t sub_of_prefix[1 << kL1Bits], prefix_of_sub[kSubTables];
 };
 
 static_assert(sizeof(StreamState) % 16 == 0, "the staging areas behind the tables take 16-byte accesses");
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ uint64_t load_le(const uint8_t* p, int bytes) {
   uint64_t v = 0;
@@ -94,7 +101,7 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   if (tid == 0) {
     int err = 0;
     S.l1 = reinterpret_cast<uint2*>(tables);
-    S.l2 = reinterpret_cast<uint2*>(tables + kTableBytes);
+    S.sub = reinterpret_cast<uint2*>(tables + kTableBytes);
     S.kraft = 0; S.count_sum = 0; S.bit_sum = 0; S.seen_max = 0; S.nused = 0; S.only_rep = 0;
     if (bytes < kHeaderBytes) {
       err = LC_ERR_FORMAT;
@@ -195,33 +202,47 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   if (S.nused < 2 && tid == 0) S.sorted_rep[0] = S.only_rep;
   __syncthreads();
 
-  // ---- lookup tables: one thread per entry, canonical decode of the entry's own index
-  for (uint32_t idx = tid; idx < (1u << kL2Bits); idx += nthreads) {
-    uint2 ent = make_uint2(0u, kLongCode);
-    if (S.nused < 2) {
-      ent = make_uint2(S.only_rep, 0u);
-    } else {
-      const uint2 r = canonical_lookup(S, idx, kL2Bits);
-      if (r.y) ent = make_uint2(S.sorted_rep[r.x], r.y);
+  // ---- lookup tables: canonical decode of each entry's own index
+  // first-level prefixes that belong to longer codes get a sub-table each, as long as there are some left
+  if (tid == 0) {
+    uint32_t next = 0;
+    for (uint32_t idx = 0; idx < (1u << kL1Bits); ++idx) {
+      uint32_t sub = kSubTables - 1;  // the "longer" sub-table
+      if (S.nused >= 2 && canonical_lookup(S, idx, kL1Bits).y == 0 && next < kSubTables - 1) {
+        sub = next++;
+        S.prefix_of_sub[sub] = (uint8_t)idx;
+      }
+      S.sub_of_prefix[idx] = (uint8_t)sub;
     }
-    S.l2[idx] = ent;
+    S.nsub = next;
   }
+  __syncthreads();
   for (uint32_t k = tid; k < (1u << kL1Bits) * kL1Rep; k += nthreads) {
-    uint2 ent = make_uint2(0u, kLongCode);
+    const uint32_t idx = k / kL1Rep;
+    uint2 ent;
     if (S.nused < 2) {
       ent = make_uint2(S.only_rep, 0u);
     } else {
-      const uint2 r = canonical_lookup(S, k / kL1Rep, kL1Bits);
+      const uint2 r = canonical_lookup(S, idx, kL1Bits);
       if (r.y) ent = make_uint2(S.sorted_rep[r.x], r.y);
+      else ent = make_uint2(smem_addr(S.sub) + S.sub_of_prefix[idx] * kSubBytes, kLongCode);
     }
     S.l1[k] = ent;
+  }
+  for (uint32_t k = tid; k < kSubTables << kSubBits; k += nthreads) {
+    const uint32_t sub = k >> kSubBits, j = k & ((1u << kSubBits) - 1);
+    uint2 ent = make_uint2(0u, kLongCode);
+    if (sub < S.nsub) {
+      const uint2 r = canonical_lookup(S, ((uint32_t)S.prefix_of_sub[sub] << kSubBits) | j, kL2Bits);
+      if (r.y) ent = make_uint2(S.sorted_rep[r.x], r.y);
+    }
+    S.sub[k] = ent;
   }
   __syncthreads();
   return 0;
 }
 
 // ---- shared-memory access by 32-bit shared address (keeps the hot loop free of generic addressing)
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
   uint32_t v;
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -259,21 +280,23 @@ struct Source {
   uint32_t slim;      // staged: shared address of the last readable word (zero slack after the chunk)
 };
 
-// Canonical search for a code longer than kL2Bits that starts at bit `bitpos` of the chunk.
-__device__ __noinline__ uint2 decode_long(const StreamState& S, const uint32_t* g, uint32_t nw, uint32_t bitpos,
-                                          int32_t* status) {
+// Table-free canonical decode of the code that starts at bit `bitpos` of a chunk in global memory
+// (the slow path for ragged or oversized chunks): {representative, length}.
+__device__ __noinline__ uint2 decode_any(const StreamState& S, const uint32_t* g, uint32_t nw, uint32_t bitpos,
+                                         int32_t* status) {
+  if (S.nused < 2) return make_uint2(S.only_rep, 0u);
   auto rd = [&](uint32_t i) { return i < nw ? __ldg(g + i) : 0u; };
   const uint32_t wi = bitpos >> 5, p = bitpos & 31;
   const unsigned long long a = ((unsigned long long)rd(wi) << 32) | rd(wi + 1);
   const unsigned long long b = rd(wi + 2);
   const unsigned long long window = p ? ((a << p) | (b >> (32 - p))) : a;
-  for (uint32_t L = kL2Bits + 1; L <= S.max_len; ++L) {
+  for (uint32_t L = 1; L <= S.max_len; ++L) {
     const unsigned long long c = window >> (64 - L);
     if (c >= S.first_code[L] && c - S.first_code[L] < S.len_count[L])
       return make_uint2(S.sorted_rep[S.len_offset[L] + (uint32_t)(c - S.first_code[L])], L);
   }
   set_status(status, LC_ERR_FORMAT);  // no code matches: damaged payload
-  return make_uint2(0u, S.max_len ? S.max_len : 1u);
+  return make_uint2(0u, S.max_len);
 }
 
 // A lane's read state in one stream of a staged chunk: `cnt` valid bits at the top of hi:lo (the bits
@@ -347,12 +370,11 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
                                                     const float* base, float* out, uint64_t c, uint32_t lane,
                                                     int32_t* status) {
   LaneBits bits[KS];
-  uint32_t l1lane[KS], l2base[KS];
+  uint32_t l1lane[KS];
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
     bits[s].seek(W[s], start[s]);
     l1lane[s] = smem_addr(S[s].l1) | ((lane & (kL1Rep - 1)) * 8u);
-    l2base[s] = smem_addr(S[s].l2);
   }
   const uint64_t e0 = c * kChunkElems + 4 * lane;
   float4 b = ldg_stream_v4(base + e0);
@@ -370,11 +392,12 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
       }
       uint2 ent[KS];
 #pragma unroll
-      for (int s = 0; s < KS; ++s) ent[s] = lds_u64(l1lane[s] | ((bits[s].hi >> kIndexShift) & kL1Mask));
+      for (int s = 0; s < KS; ++s) ent[s] = lds_u64(l1lane[s] | ((bits[s].hi >> kL1Shift) & kL1Mask));
       uint32_t longest = 0;
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        lds_u64_if_long(ent[s], l2base[s] | ((bits[s].hi >> kIndexShift) & kL2Mask));
+        // where the first level says "longer", ent.x is the shared address of the prefix's sub-table
+        lds_u64_if_long(ent[s], ent[s].x | ((bits[s].hi >> kSubShift) & kSubMask));
         longest |= ent[s].y;  // lengths are < 64, the marker is all ones
       }
       if (__any_sync(0xffffffffu, longest > 63u)) {
@@ -417,8 +440,8 @@ __device__ __noinline__ void decode_chunk_global(const StreamState* S, GlobalChu
         const uint32_t w0 = wi < G.nw[s] ? __ldg(G.g[s] + wi) : 0u;
         const uint32_t w1 = wi + 1 < G.nw[s] ? __ldg(G.g[s] + wi + 1) : 0u;
         const uint32_t peek = __funnelshift_l(w1, w0, sh);
-        uint2 ent = S[s].l2[peek >> (32 - kL2Bits)];
-        if (ent.y > 63u) ent = decode_long(S[s], G.g[s], G.nw[s], pos[s], status);
+        (void)peek;
+        const uint2 ent = decode_any(S[s], G.g[s], G.nw[s], pos[s], status);
         x = __fadd_rn(x, __uint_as_float(ent.x));
         pos[s] += ent.y;
       }
