@@ -44,15 +44,9 @@ constexpr uint32_t kSubBytes = (1u << kSubBits) * 8;
 constexpr uint32_t kLongCode = 0xFFFFFFFFu;
 static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill guarantee");
 
-// The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory, so that an
-// entry's address is (table base | index bits), one logic operation, with both index fields taken from
-// the same shifted copy of the bit buffer.
+// The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory.
 constexpr uint32_t kTableBytes = 8192;
 static_assert((1 << kL1Bits) * kL1Rep * 8 == kTableBytes && kSubTables * kSubBytes == kTableBytes, "table sizes");
-constexpr uint32_t kL1Mask = ((1u << kL1Bits) - 1) << 7;    // index * 128 bytes (16 copies of 8 bytes)
-constexpr int kL1Shift = 32 - kL1Bits - 7;                  // (hi >> 19) & kL1Mask == first-level index * 128
-constexpr uint32_t kSubMask = ((1u << kSubBits) - 1) << 3;  // index * 8 bytes
-constexpr int kSubShift = 32 - kL1Bits - kSubBits - 3;      // (hi >> 17) & kSubMask == sub-table index * 8
 
 struct alignas(16) StreamState {
   uint2* l1;  // [(1 << kL1Bits) * kL1Rep] {bit pattern of rep, code length}; length kLongCode = not resolved here
@@ -248,11 +242,6 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
   asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ uint2 lds_u64(uint32_t addr) {
-  uint2 v;
-  asm("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-  return v;
-}
 // Streaming 16-byte load; volatile so that it stays where it is written (early in the loop body).
 __device__ __forceinline__ float4 ldg_stream_v4(const float* p) {
   float4 v;
@@ -264,12 +253,29 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-// Second-level lookup for the lanes whose first-level entry says "longer code": one predicated load,
-// so that the few lanes that need it do not turn the warp's symbol step into a divergent branch.
-__device__ __forceinline__ void lds_u64_if_long(uint2& ent, uint32_t addr) {
-  asm("{\n\t.reg .pred q;\n\tsetp.gt.u32 q, %1, 63;\n\t@q ld.shared.v2.u32 {%0,%1}, [%2];\n\t}"
-      : "+r"(ent.x), "+r"(ent.y)
-      : "r"(addr));
+// Two-level table lookup of the code at the top of `hi`: {representative, length}, length kLongCode if
+// the code is longer than kL2Bits. `l1lane` = shared address of this lane's copy of first-level entry 0.
+// The first-level entry of a prefix that belongs to longer codes holds the shared address of the
+// prefix's sub-table, which is read by a predicated load (no branch for the few lanes that need it).
+// Written in PTX so that index scaling and base addition stay multiply-adds (they then run beside the
+// shifts and compares instead of competing with them for the integer pipe).
+__device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane) {
+  uint2 ent;
+  asm("{\n\t"
+      ".reg .u32 t, a;\n\t"
+      ".reg .pred q;\n\t"
+      "shr.u32 t, %2, %4;\n\t"
+      "mad.lo.u32 a, t, %5, %3;\n\t"
+      "ld.shared.v2.u32 {%0,%1}, [a];\n\t"
+      "setp.gt.u32 q, %1, 63;\n\t"
+      "shl.b32 t, %2, %6;\n\t"
+      "shr.u32 t, t, %7;\n\t"
+      "mad.lo.u32 a, t, 8, %0;\n\t"
+      "@q ld.shared.v2.u32 {%0,%1}, [a];\n\t"
+      "}"
+      : "=&r"(ent.x), "=&r"(ent.y)
+      : "r"(hi), "r"(l1lane), "n"(32 - kL1Bits), "n"(kL1Rep * 8), "n"(kL1Bits), "n"(32 - kSubBits));
+  return ent;
 }
 
 // Where a chunk's words are read from.
@@ -391,13 +397,10 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
         for (int s = 0; s < KS; ++s) bits[s].refill(W[s].slim);
       }
       uint2 ent[KS];
-#pragma unroll
-      for (int s = 0; s < KS; ++s) ent[s] = lds_u64(l1lane[s] | ((bits[s].hi >> kL1Shift) & kL1Mask));
       uint32_t longest = 0;
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        // where the first level says "longer", ent.x is the shared address of the prefix's sub-table
-        lds_u64_if_long(ent[s], ent[s].x | ((bits[s].hi >> kSubShift) & kSubMask));
+        ent[s] = lookup_code(bits[s].hi, l1lane[s]);
         longest |= ent[s].y;  // lengths are < 64, the marker is all ones
       }
       if (__any_sync(0xffffffffu, longest > 63u)) {
