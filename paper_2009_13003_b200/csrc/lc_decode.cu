@@ -42,6 +42,7 @@ constexpr int kL2Bits = kL1Bits + kSubBits;        // longest code the two table
 constexpr int kSubTables = 16;                     // 15 usable + one that only says "longer"
 constexpr uint32_t kSubBytes = (1u << kSubBits) * 8;
 constexpr uint32_t kLongCode = 0xFFFFFFFFu;
+constexpr uint32_t kOverrunBytes = 512;  // padding behind the last staging area (see LaneBits::refill)
 static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill guarantee");
 
 // The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory.
@@ -319,26 +320,26 @@ struct LaneBits {
     hi = __funnelshift_l(w1, w0, sh);
     lo = w1 << sh;
     cnt = 64 - (int)sh;
-    next = at + 8u;
+    next = min(at + 8u, W.slim);
   }
   // Tops the buffer up with one word if 32 bits or fewer are left; afterwards cnt >= 33. All predicated.
-  __device__ __forceinline__ void refill(uint32_t slim) {
+  // The load is not clamped: between two seeks (which do clamp) `next` moves by at most 64 words, and the
+  // kernel's shared memory ends with kOverrunBytes of padding, so a damaged stream can make a lane read
+  // stale shared memory but never leave the allocation.
+  __device__ __forceinline__ void refill() {
     asm volatile(
         "{\n\t"
         ".reg .pred q;\n\t"
-        ".reg .u32 w, t, a;\n\t"
+        ".reg .u32 w, t;\n\t"
         "setp.le.s32 q, %2, 32;\n\t"
-        "min.u32 a, %3, %4;\n\t"
-        "@q ld.shared.u32 w, [a];\n\t"
-        "@q shf.r.clamp.b32 t, w, 0, %2;\n\t"   // w >> cnt (0 when cnt == 32)
+        "@q ld.shared.u32 w, [%3];\n\t"
+        "@q shf.r.clamp.b32 t, w, 0, %2;\n\t"   // high word of (w:0) >> cnt, i.e. w >> cnt (0 when cnt == 32)
         "@q or.b32 %0, %0, t;\n\t"
-        "@q sub.s32 t, 32, %2;\n\t"
-        "@q shf.l.clamp.b32 %1, 0, w, t;\n\t"   // lo was 0: lo = w << (32 - cnt) (0 when cnt == 0)
+        "@q shf.r.clamp.b32 %1, 0, w, %2;\n\t"  // low word of (w:0) >> cnt; lo was 0 because cnt <= 32
         "@q add.s32 %2, %2, 32;\n\t"
         "@q add.u32 %3, %3, 4;\n\t"
         "}"
-        : "+r"(hi), "+r"(lo), "+r"(cnt), "+r"(next)
-        : "r"(slim));
+        : "+r"(hi), "+r"(lo), "+r"(cnt), "+r"(next));
   }
   __device__ __forceinline__ void consume(uint32_t len) {
     hi = __funnelshift_l(lo, hi, len);
@@ -394,7 +395,7 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
     for (int e = 0; e < 4; ++e) {
       if ((e & 1) == 0) {
 #pragma unroll
-        for (int s = 0; s < KS; ++s) bits[s].refill(W[s].slim);
+        for (int s = 0; s < KS; ++s) bits[s].refill();
       }
       uint2 ent[KS];
       uint32_t longest = 0;
@@ -553,13 +554,14 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
                              int32_t* status, cudaStream_t cs) {
   static int sms = 0;
   constexpr uint32_t kTables = kTableBytes + KS * (2 * kTableBytes + sizeof(StreamState));
-  constexpr uint32_t kMaxDyn = kSmemPerSm - 1024;  // leave room for the static __shared__ variables
+  constexpr uint32_t kMaxDyn = kSmemPerSm - 1024 - kOverrunBytes;  // room for static __shared__ and the padding
   if (sms == 0) {
     int dev = 0, v = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDyn);
+    e = cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(kMaxDyn + kOverrunBytes));
     if (e != cudaSuccess) return e;
     sms = v;
   }
@@ -577,7 +579,7 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
   while (warps > 8 && kTables + (uint64_t)warps * KS * want_stage > kMaxDyn) warps -= 4;
   uint32_t stage = ((kMaxDyn - kTables) / (warps * KS)) / 16 * 16;
   if (stage > kChunkElems * 8 + 16) stage = kChunkElems * 8 + 16;
-  const uint32_t dyn = kTables + warps * KS * stage;
+  const uint32_t dyn = kTables + warps * KS * stage + kOverrunBytes;
   uint64_t want = (nchunks + warps - 1) / warps;
   if (want == 0) want = 1;  // still validates the streams
   const unsigned grid = (unsigned)(want < (uint64_t)sms ? want : (uint64_t)sms);
