@@ -12,8 +12,7 @@ bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p
 struct Carved {
   Control* ctl;
   unsigned long long* tiles;
-  uint8_t* eplane;
-  uint32_t* splane;
+  uint8_t* plane;
 };
 
 Carved carve(void* workspace, const WorkspaceLayout& W) {
@@ -21,8 +20,7 @@ Carved carve(void* workspace, const WorkspaceLayout& W) {
   Carved c;
   c.ctl = reinterpret_cast<Control*>(w + W.control_off);
   c.tiles = reinterpret_cast<unsigned long long*>(w + W.tiles_off);
-  c.eplane = w + W.eplane_off;
-  c.splane = reinterpret_cast<uint32_t*>(w + W.splane_off);
+  c.plane = w + W.plane_off;
   return c;
 }
 
@@ -65,11 +63,11 @@ int lc_compress(const float* base, const float* cur, uint64_t n, int nbits, void
   const Carved c = carve(workspace, W);
 
   // control block and tile descriptors start at zero
-  cudaError_t e = cudaMemsetAsync(workspace, 0, W.eplane_off, cs);
+  cudaError_t e = cudaMemsetAsync(workspace, 0, W.plane_off, cs);
   if (e != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_stats(base, cur, n, c.ctl, c.eplane, c.splane, cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_encode(c.ctl, c.tiles, c.eplane, c.splane, n, static_cast<uint8_t*>(stream), cs)) != cudaSuccess)
+  if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), cs)) != cudaSuccess)
     return LC_ERR_CUDA;
   return LC_OK;
 }
@@ -88,13 +86,13 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
   cudaEvent_t ev[4];
   for (int i = 0; i < 4; ++i)
     if (cudaEventCreate(&ev[i]) != cudaSuccess) return LC_ERR_CUDA;
-  bool ok = cudaMemsetAsync(workspace, 0, W.eplane_off, cs) == cudaSuccess;
+  bool ok = cudaMemsetAsync(workspace, 0, W.plane_off, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[0], cs) == cudaSuccess;
-  ok = ok && launch_stats(base, cur, n, c.ctl, c.eplane, c.splane, cs) == cudaSuccess;
+  ok = ok && launch_stats(base, cur, n, c.ctl, c.plane, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[1], cs) == cudaSuccess;
   ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[2], cs) == cudaSuccess;
-  ok = ok && launch_encode(c.ctl, c.tiles, c.eplane, c.splane, n, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
+  ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[3], cs) == cudaSuccess;
   ok = ok && cudaEventSynchronize(ev[3]) == cudaSuccess;
   for (int i = 0; ok && i < 3; ++i) ok = cudaEventElapsedTime(&kernel_ms[i], ev[i], ev[i + 1]) == cudaSuccess;

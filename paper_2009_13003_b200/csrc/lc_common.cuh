@@ -35,19 +35,20 @@ __host__ __device__ inline StreamLayout stream_layout(uint64_t n, uint32_t nsym)
 }
 
 // ---- statistics pass -> encode pass hand-over ("key plane") -----------------------------------
-// The statistics kernel leaves, for every element, its exponent field (1 byte) and its sign (1 bit)
-// in the workspace so that the encode pass reads 1.125 bytes per element instead of 8.
+// The statistics kernel leaves one byte per element in the workspace so that the encode pass reads
+// 1 byte per element instead of 8: (sign << 7) | (exponent field & 127). That identifies the bucket as
+// long as every exponent field is below 128, i.e. every |delta| < 2; if some delta is larger (the
+// statistics tell), the encode pass ignores the plane and recomputes the keys from base and cur.
 // A *unit* is 1024 consecutive elements = 8 steps of one chunk, handled by one warp iteration:
-//   exponent plane, unit u: bytes [1024u, 1024u+1024): byte 512*(r/4) + 16*lane + 4*(r%4) + e
-//   sign plane, unit u: u32 word 32u + lane, bit 31 - (4r + e)
+//   unit u: bytes [1024u, 1024u+1024): byte 512*(r/4) + 16*lane + 4*(r%4) + e
 // for step r (0..7) of the unit, lane (0..31) and slot e (0..3), i.e. element 1024u + 128r + 4lane + e.
 constexpr uint32_t kUnitElems = 1024;
 constexpr uint32_t kUnitsPerChunk = kChunkElems / kUnitElems;
 
-// ---- encode pass tiling --------------------------------------------------------------------------
-constexpr uint32_t kEncWarps = 8;  // chunks per tile (one per warp)
+// ---- encode pass ----------------------------------------------------------------------------------
+constexpr uint32_t kEncWarps = 8;  // warps per CTA of the encode pass (one chunk per warp at a time)
 
-// Tile descriptor of the decoupled look-back scan: flag in the top two bits, bytes below.
+// Chunk descriptor of the decoupled look-back scan of the encode pass: flag in the top two bits, bytes below.
 constexpr uint64_t kTileFlagShift = 62;
 constexpr uint64_t kTileInvalid = 0, kTileAggregate = 1, kTilePrefix = 2, kTileAbort = 3;
 constexpr uint64_t kTileValueMask = (1ull << kTileFlagShift) - 1;
@@ -63,11 +64,13 @@ struct EncEntry {
 // Control block at the start of the workspace. Zeroed at the start of every lc_compress.
 struct Control {
   int32_t status;         // first device-detected error, 0 if none
-  uint32_t ticket;        // next encode tile
+  uint32_t ticket;        // next chunk of the encode pass
   uint32_t nsym;          // written by the table kernel
   uint32_t max_len;       // written by the table kernel
   uint64_t payload_bits;  // written by the table kernel
-  uint64_t pad_[29];
+  uint32_t wide;          // written by the table kernel: some delta has an exponent field >= 128
+  uint32_t pad32_;
+  uint64_t pad_[28];
   unsigned long long count[kKeys];  // elements per key
   uint32_t inv_min[kKeys];          // max over the bucket of ~bits (zero-initialised running minimum)
   uint32_t max_bits[kKeys];         // max over the bucket of bits
@@ -76,20 +79,18 @@ struct Control {
 static_assert(sizeof(Control) % 256 == 0, "control block must keep the planes 256-byte aligned");
 
 struct WorkspaceLayout {
-  uint64_t control_off, tiles_off, eplane_off, splane_off, total;
-  uint64_t ntiles, nunits;
+  uint64_t control_off, tiles_off, plane_off, total;
+  uint64_t nchunks, nunits;
 };
 
 __host__ __device__ inline WorkspaceLayout workspace_layout(uint64_t n) {
   WorkspaceLayout W;
-  const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
-  W.ntiles = (nchunks + kEncWarps - 1) / kEncWarps;
-  W.nunits = nchunks * kUnitsPerChunk;
+  W.nchunks = (n + kChunkElems - 1) / kChunkElems;
+  W.nunits = W.nchunks * kUnitsPerChunk;
   W.control_off = 0;
-  W.tiles_off = sizeof(Control);
-  W.eplane_off = align_up(W.tiles_off + 8 * W.ntiles, 256);
-  W.splane_off = W.eplane_off + nchunks * kChunkElems;          // 1 byte per element, whole chunks
-  W.total = align_up(W.splane_off + nchunks * (kChunkElems / 8), 256);  // 1 bit per element
+  W.tiles_off = sizeof(Control);                                // one 8-byte descriptor per chunk
+  W.plane_off = align_up(W.tiles_off + 8 * W.nchunks, 256);
+  W.total = align_up(W.plane_off + W.nchunks * kChunkElems, 256);  // 1 byte per element, whole chunks
   return W;
 }
 
@@ -97,11 +98,11 @@ __host__ __device__ inline WorkspaceLayout workspace_layout(uint64_t n) {
 __device__ inline void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
 
 // ---- launchers (each defined next to its kernel) ---------------------------------------------------
-cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* eplane,
-                         uint32_t* splane, cudaStream_t cs);
+cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
+                         cudaStream_t cs);
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, cudaStream_t cs);
-cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* eplane,
-                          const uint32_t* splane, uint64_t n, uint8_t* stream, cudaStream_t cs);
+cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
+                          const float* cur, uint64_t n, uint8_t* stream, cudaStream_t cs);
 
 struct DecodeStreams {
   const uint8_t* ptr[4];

@@ -4,42 +4,68 @@
 // indices, is Huffman-coded). Element order, bit order and the two indices are those of the stream
 // format text, sections 2 and 3.
 //
-// One warp codes one chunk of 4096 elements; lane t owns lane sub-stream t. Per chunk:
-//   A. every lane sums the code lengths of its 128 elements            -> lane index, chunk size
-//   B. the chunk's bits are assembled in a warp-private shared-memory staging area (every lane ORs its
-//      words in at its bit offset, found with a warp shuffle scan of the lane lengths)
-//   C. the chunk's byte offset comes from an exclusive scan over all chunks, done across CTAs with a
-//      decoupled look-back over per-tile descriptors (a tile = the 8 chunks of one CTA iteration);
-//   D. the staged chunk is copied to the payload with coalesced 16-byte stores.
-// Tiles are handed out by an atomic ticket, so every tile a CTA waits for has already been started by
-// a running CTA. The wait is bounded all the same: after kSpinLimit polls the CTA records
+// A CTA takes a tile of 8 consecutive chunks, one per warp; lane t owns lane sub-stream t. Per chunk:
+//   A. every lane codes its 128 elements into its own column of a warp-private word matrix in shared
+//      memory (word k of lane t at k*32 + t: plain stores, no bank conflicts, no atomics). Code and
+//      length come packed in one 32-bit table entry (a 16-byte entry made the lookups saturate the
+//      shared-memory pipe); the rare codes of 27..32 bits are fetched by a predicated second load.
+//      Emitting a finished word is a handful of predicated instructions;
+//   B. a warp shuffle scan of the lane bit counts gives every lane its bit offset in the chunk (the
+//      lane index of the stream) and the chunk its size, which is published at once;
+//   C. the lanes' words are shifted to their bit offsets and ORed into the chunk image (shared memory);
+//   D. the tile's byte offset comes from an exclusive scan over all tiles, done across CTAs with a
+//      decoupled look-back over per-tile descriptors (per-chunk descriptors were tried: with thousands
+//      of chunks in flight every look-back walks too far back);
+//   E. the chunk image is copied to the payload with coalesced 16-byte stores.
+// Tiles are handed out by an atomic ticket, so every tile a CTA waits for in D has already been
+// started by a running CTA. The wait is bounded all the same: after kSpinLimit polls the CTA records
 // LC_ERR_TIMEOUT, marks its tile aborted (successors see that at once and abort too) and moves on.
 //
-// Bound: reads 1.125 bytes and writes about 0.5 bytes per element, so this pass is limited by the
-// integer work per element, not by HBM.
+// Rare cases take a compact two-pass path (lengths, then bits ORed in place): the ragged last chunk,
+// codes longer than 32 bits, a lane or chunk that outgrows its shared-memory area, and vectors with an
+// exponent field >= 128, for which the one-byte key plane is not enough and keys come from base and cur.
+//
+// Bound: reads 1 byte and writes about 0.5 bytes per element, so this pass is limited by the integer
+// work per element, not by HBM.
 #include "lc_common.cuh"
 
 namespace lc {
 namespace {
 
 constexpr int kEncThreads = kEncWarps * 32;
-constexpr uint32_t kStageWords = 1536;  // per warp: 6 KB = 12 bits per element on average
-constexpr uint32_t kEncSmem = kEncWarps * kStageWords * 4;
+// 48 KB of dynamic shared memory per CTA (four CTAs per SM), split evenly between the warps that work:
+// all 8 while an average chunk fits half of a 6 KB share (column matrix + chunk image), else 4, 2 or 1.
+constexpr uint32_t kEncSmem = 48 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 20;
 
+constexpr uint32_t kPackedLenShift = 26;                      // packed entry: length << 26 | code
+constexpr uint32_t kPackedCodeMask = (1u << kPackedLenShift) - 1;
+constexpr uint32_t kPackedLong = 63;                          // length field of a code that does not fit
+
 struct Tables {
-  uint2 enc[kKeys];       // {code_lo, len}
-  uint32_t enc_hi[kKeys];
+  uint32_t packed[256];  // by plane byte: length << 26 | code for codes of up to 26 bits, else length field 63
+  uint2 full[256];       // by plane byte: {code, length} for codes of up to 32 bits
 };
 
-// Index into the encode table of slot e of a row: exponent byte e of `word`, sign from bit (3 - e) of
-// the row's sign nibble.
-__device__ __forceinline__ uint32_t key_of(uint32_t word, uint32_t nibble, int e) {
-  return ((word >> (8 * e)) & 255u) | (((nibble >> (3 - e)) & 1u) << 8);
-}
+// Where the slow path gets an element's key from.
+struct KeySource {
+  const uint8_t* plane;  // used unless `wide`
+  const float* base;
+  const float* cur;
+  bool wide;
+  __device__ __forceinline__ uint32_t key(uint64_t c, uint32_t j, uint32_t lane, uint32_t e) const {
+    if (wide) {
+      const uint64_t i = c * kChunkElems + 128ull * j + 4 * lane + e;
+      return __float_as_uint(__fsub_rn(cur[i], base[i])) >> 23;
+    }
+    const uint32_t b = plane[c * kChunkElems + (j >> 2) * 512 + lane * 16 + (j & 3) * 4 + e];
+    return ((b & 128u) << 1) | (b & 127u);
+  }
+};
 
-// Appends a code of at most 32 bits to the lane's bit accumulator and emits completed 32-bit words.
-struct Packer {
+// Appends a code of at most 32 bits to the lane's bit accumulator and ORs completed 32-bit words into the
+// chunk image at `dst` (shared or global memory).
+struct OrPacker {
   unsigned long long acc;  // pending bits in the low `nb` bits
   uint32_t nb;
   uint32_t* dst;  // next word of the chunk this lane touches
@@ -57,30 +83,25 @@ struct Packer {
   }
 };
 
-// Slow, compact path for the three rare cases: the ragged last chunk, codes longer than 32 bits, and
-// a chunk too large for the staging area. Reads the plane from global memory element by element.
-// With dst == nullptr it only returns the lane's bit count.
-__device__ __noinline__ uint32_t chunk_slow(const Tables& tb, const uint8_t* __restrict__ eplane,
-                                            const uint32_t* __restrict__ splane, uint64_t c, uint32_t lane,
+// Slow, compact path (see the header). With dst == nullptr it only returns the lane's bit count;
+// otherwise it ORs the lane's bits into the zeroed chunk image at dst, starting at bit lane_start.
+__device__ __noinline__ uint32_t chunk_slow(const EncEntry* __restrict__ enc, KeySource ks, uint64_t c, uint32_t lane,
                                             uint64_t n, uint32_t* dst, uint32_t lane_start) {
-  Packer pk{0ull, lane_start & 31u, dst ? dst + (lane_start >> 5) : nullptr};
+  OrPacker pk{0ull, lane_start & 31u, dst ? dst + (lane_start >> 5) : nullptr};
   uint32_t bits = 0;
   for (uint32_t j = 0; j < kSteps; ++j) {
-    const uint32_t sw = splane[c * 128 + (j >> 3) * 32 + lane];
     for (uint32_t e = 0; e < kGroup; ++e) {
       const uint64_t i = c * kChunkElems + 128ull * j + 4 * lane + e;
       if (i >= n) continue;
-      const uint32_t E = eplane[c * kChunkElems + (j >> 2) * 512 + lane * 16 + (j & 3) * 4 + e];
-      const uint32_t s = (sw >> (31 - ((j & 7) * 4 + e))) & 1u;
-      const uint32_t key = E | (s << 8);
-      const uint2 en = tb.enc[key];
-      bits += en.y;
+      const uint32_t key = ks.key(c, j, lane, e);
+      const EncEntry en = enc[key];
+      bits += en.len;
       if (dst) {
-        if (en.y > 32) {
-          pk.put(tb.enc_hi[key], en.y - 32);
-          pk.put(en.x, 32);
+        if (en.len > 32) {
+          pk.put(en.code_hi, en.len - 32);
+          pk.put(en.code_lo, 32);
         } else {
-          pk.put(en.x, en.y);
+          pk.put(en.code_lo, en.len);
         }
       }
     }
@@ -96,11 +117,41 @@ __device__ __forceinline__ void st_tile(unsigned long long* p, unsigned long lon
   *reinterpret_cast<volatile unsigned long long*>(p) = v;
 }
 
-__global__ void __launch_bounds__(kEncThreads)
-encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
-              const uint8_t* __restrict__ eplane, const uint32_t* __restrict__ splane, uint64_t n,
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Fast-path state of a lane: pending bits in hi:lo (low `nb` bits valid), next word slot in its column.
+struct ColumnPacker {
+  uint32_t hi, lo, nb;
+  uint32_t dst;  // shared address of the next word of this lane's column (stride 128 bytes)
+  uint32_t lim;  // shared address one past the column
+  __device__ __forceinline__ void put(uint32_t code, uint32_t len) {
+    // (hi:lo) = (hi:lo) << len | code, len <= 32
+    hi = __funnelshift_lc(lo, hi, len);
+    lo = __funnelshift_lc(0u, lo, len) | code;
+    nb += len;
+    // emit the oldest 32 pending bits once there are 32 or more, unless the column is full
+    asm volatile(
+        "{\n\t"
+        ".reg .pred q;\n\t"
+        ".reg .u32 w;\n\t"
+        "setp.ge.u32 q, %0, 32;\n\t"
+        "setp.lt.and.u32 q, %1, %4, q;\n\t"
+        "@q sub.u32 %0, %0, 32;\n\t"
+        "@q shf.r.clamp.b32 w, %3, %2, %0;\n\t"
+        "@q st.shared.u32 [%1], w;\n\t"
+        "@q add.u32 %1, %1, 128;\n\t"
+        "}"
+        : "+r"(nb), "+r"(dst)
+        : "r"(hi), "r"(lo), "r"(lim)
+        : "memory");
+  }
+};
+
+__global__ void __launch_bounds__(kEncThreads, 4)
+encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles, const uint8_t* __restrict__ plane,
+              const float* __restrict__ base, const float* __restrict__ cur, uint64_t n,
               uint8_t* __restrict__ stream) {
-  extern __shared__ __align__(16) uint32_t s_stage_all[];
+  extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ Tables tb;
   __shared__ uint32_t s_chunk_bytes[kEncWarps];
   __shared__ uint32_t s_tile;
@@ -110,23 +161,69 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
   if (ctl->status != 0) return;  // the table pass rejected the vector
 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (uint32_t k = tid; k < kKeys; k += kEncThreads) {
-    const EncEntry e = ctl->enc[k];
-    tb.enc[k] = make_uint2(e.code_lo, e.len);
-    tb.enc_hi[k] = e.code_hi;
+  for (uint32_t b = tid; b < 256; b += kEncThreads) {
+    const EncEntry e = ctl->enc[((b & 128u) << 1) | (b & 127u)];
+    tb.full[b] = make_uint2(e.code_lo, e.len);
+    tb.packed[b] = e.len <= kPackedLenShift ? (e.len << kPackedLenShift) | e.code_lo : kPackedLong << kPackedLenShift;
   }
+  __syncthreads();
+
   const uint32_t nsym = ctl->nsym;
   const bool long_codes = ctl->max_len > 32;
+  const KeySource ks{plane, base, cur, ctl->wide != 0};
   const StreamLayout L = stream_layout(n, nsym);
   const uint64_t nchunks = L.nchunks;
-  const uint64_t ntiles = (nchunks + kEncWarps - 1) / kEncWarps;
   unsigned long long* chunk_index = reinterpret_cast<unsigned long long*>(stream + L.chunk_index_off);
   uint16_t* lane_index = reinterpret_cast<uint16_t*>(stream + L.lane_index_off);
   uint8_t* payload = stream + L.payload_off;
-  uint32_t* stage = s_stage_all + warp * kStageWords;
+  // how many warps work: as many as can each hold an average chunk (plus 15 %) twice
+  const uint64_t avg_bytes = nchunks ? ctl->payload_bits / 8 / nchunks : 0;
+  const uint64_t need = avg_bytes + avg_bytes / 7 + 64;
+  uint32_t active = kEncWarps;
+  while (active > 1 && need > kEncSmem / active / 2) active >>= 1;
+  const uint32_t image_words = kEncSmem / active / 8;  // half of the warp's share, in words
+  const uint32_t lane_words = image_words / 32;        // rows of the column matrix
+  uint32_t* column = s_dyn + (warp % active) * (2 * image_words);  // word k of lane t at column[k*32 + t]
+  uint32_t* image = column + image_words;
+  const uint32_t packed_addr = smem_addr(tb.packed);
+
+  // Packed table entries of the four plane bytes of `word`.
+  auto lookup4 = [&](uint32_t word, uint32_t (&g)[4]) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint32_t b = __byte_perm(word, 0u, 0x4440 + e);  // plane byte of slot e
+      // volatile: keeps the loads where they are written, one row ahead of their use
+      asm volatile("ld.shared.u32 %0, [%1];" : "=r"(g[e]) : "r"(packed_addr + b * 4u));
+    }
+  };
+  // Appends the four codes of `word`, whose packed entries are g. Only the marker has bit 31 set (packed
+  // lengths are <= 26), so one test per row finds the rare codes of 27..32 bits, which come from `full`.
+  auto put4 = [&](ColumnPacker& pk, uint32_t word, const uint32_t (&g)[4]) {
+    uint32_t code[4], len[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      len[e] = g[e] >> kPackedLenShift;
+      code[e] = g[e] & kPackedCodeMask;
+    }
+    if (__any_sync(0xffffffffu, (int)(g[0] | g[1] | g[2] | g[3]) < 0)) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if ((int)g[e] < 0) {
+          const uint2 f = tb.full[__byte_perm(word, 0u, 0x4440 + e)];
+          code[e] = f.x;
+          len[e] = f.y;
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) pk.put(code[e], len[e]);
+  };
+  auto fast_chunk = [&](uint64_t cc) { return cc < nchunks && (cc + 1) * kChunkElems <= n && !long_codes && !ks.wide; };
+
+  const uint64_t ntiles = (nchunks + active - 1) / active;
 
   while (true) {
-    __syncthreads();  // previous iteration is done with s_tile, s_chunk_bytes and the staging areas
+    __syncthreads();  // previous tile is done with s_tile, s_chunk_bytes and the shared areas
     if (tid == 0) {
       s_tile = atomicAdd(&ctl->ticket, 1u);
       s_abort = 0;
@@ -134,39 +231,44 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     __syncthreads();
     const uint64_t tile = s_tile;
     if (tile >= ntiles) break;
-    const uint64_t c = tile * kEncWarps + warp;
-    const bool valid = c < nchunks;
-    const bool full = valid && (c + 1) * kChunkElems <= n;
-    const bool fast = full && !long_codes;
+    const uint64_t c = tile * active + warp;
+    const bool valid = warp < active && c < nchunks;
+    bool fast = valid && fast_chunk(c);
 
-    // ---- load the chunk's slice of the key plane: 128 exponent bytes and 128 sign bits per lane
-    uint4 ev[8];
-    uint32_t sg[4];
-    if (fast) {
-      const uint4* ep = reinterpret_cast<const uint4*>(eplane + c * kChunkElems) + lane;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) ev[q] = __ldg(ep + 32 * q);
-#pragma unroll
-      for (int g = 0; g < 4; ++g) sg[g] = __ldg(splane + c * 128 + g * 32 + lane);
-    }
-
-    // ---- A: lane bit counts
+    // ---- A: code the lane's elements into its column. Lookups run one row (4 elements) ahead of the
+    // appends, which depend on each other through the bit accumulator.
     uint32_t lane_bits = 0;
     if (fast) {
-#pragma unroll
+      const uint4* ep = reinterpret_cast<const uint4*>(plane + c * kChunkElems) + lane;
+      const uint32_t col0 = smem_addr(column) + lane * 4;
+      ColumnPacker pk{0u, 0u, 0u, col0, col0 + lane_words * 128};
+      uint32_t g0[4], g1[4];
+      uint4 cur4 = __ldg(ep);
+      lookup4(cur4.x, g0);
+#pragma unroll 1
       for (int q = 0; q < 8; ++q) {
-        const uint32_t w[4] = {ev[q].x, ev[q].y, ev[q].z, ev[q].w};
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int j = 4 * q + r;
-          const uint32_t nib = (sg[j >> 3] >> (28 - 4 * (j & 7))) & 15u;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) lane_bits += tb.enc[key_of(w[r], nib, e)].y;
-        }
+        const uint4 nxt = __ldg(ep + 32 * (q + 1 < 8 ? q + 1 : q));  // next 16 plane bytes, one step ahead
+        lookup4(cur4.y, g1);
+        put4(pk, cur4.x, g0);
+        lookup4(cur4.z, g0);
+        put4(pk, cur4.y, g1);
+        lookup4(cur4.w, g1);
+        put4(pk, cur4.z, g0);
+        lookup4(nxt.x, g0);  // first row of the next step (unused after the last step)
+        put4(pk, cur4.w, g1);
+        cur4 = nxt;
       }
-    } else if (valid) {
-      lane_bits = chunk_slow(tb, eplane, splane, c, lane, n, nullptr, 0);
+      const bool overflow = pk.nb >= 32 || (pk.nb > 0 && pk.dst >= pk.lim);
+      if (__any_sync(0xffffffffu, overflow)) {
+        fast = false;  // some lane outgrew its column: redo the chunk the slow way
+      } else {
+        if (pk.nb > 0) column[((pk.dst - col0) >> 7) * 32 + lane] = pk.lo << (32 - pk.nb);
+        lane_bits = ((pk.dst - col0) >> 7) * 32 + pk.nb;
+      }
     }
+    if (!fast && valid) lane_bits = chunk_slow(ctl->enc, ks, c, lane, n, nullptr, 0);
+
+    // ---- B: lane offsets, lane index, chunk size; the tile's size is published as early as possible
     if (valid) lane_index[c * kLanes + lane] = (uint16_t)lane_bits;
     uint32_t incl = lane_bits;
 #pragma unroll
@@ -177,11 +279,9 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     const uint32_t lane_start = incl - lane_bits;
     const uint32_t chunk_bits = __shfl_sync(0xffffffffu, incl, 31);
     const uint32_t chunk_bytes = valid ? (uint32_t)align_up((chunk_bits + 7) / 8, kPayloadAlign) : 0u;
-    const bool staged = chunk_bytes <= kStageWords * 4;
+    const bool staged = chunk_bytes <= image_words * 4;
     if (lane == 0) s_chunk_bytes[warp] = chunk_bytes;
     __syncthreads();
-
-    // ---- publish this tile's size as early as possible
     unsigned long long tile_bytes = 0;
 #pragma unroll
     for (int w = 0; w < (int)kEncWarps; ++w) tile_bytes += s_chunk_bytes[w];
@@ -191,34 +291,28 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
       if (tile == 0) s_tile_base = 0;
     }
 
-    // ---- B: assemble the chunk in shared memory
+    // ---- C: assemble the chunk image in shared memory
     if (valid && staged) {
-      uint4* st4 = reinterpret_cast<uint4*>(stage);
-      for (uint32_t k = lane; k < chunk_bytes / 16; k += 32) st4[k] = make_uint4(0, 0, 0, 0);
+      uint4* im4 = reinterpret_cast<uint4*>(image);
+      for (uint32_t k = lane; k < chunk_bytes / 16; k += 32) im4[k] = make_uint4(0, 0, 0, 0);
       __syncwarp();
       if (fast) {
-        Packer pk{0ull, lane_start & 31u, stage + (lane_start >> 5)};
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const uint32_t w[4] = {ev[q].x, ev[q].y, ev[q].z, ev[q].w};
-#pragma unroll
-          for (int r = 0; r < 4; ++r) {
-            const int j = 4 * q + r;
-            const uint32_t nib = (sg[j >> 3] >> (28 - 4 * (j & 7))) & 15u;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const uint2 en = tb.enc[key_of(w[r], nib, e)];
-              pk.put(en.x, en.y);
-            }
-          }
+        const uint32_t nw = (lane_bits + 31) >> 5, r = lane_start & 31;
+        uint32_t* out = image + (lane_start >> 5);
+        uint32_t prev = 0;
+        for (uint32_t k = 0; k < nw; ++k) {
+          const uint32_t w = column[k * 32 + lane];
+          atomicOr(out + k, __funnelshift_r(w, prev, r));
+          prev = w;
         }
-        pk.flush();
+        const uint32_t tail = r ? prev << (32 - r) : 0u;
+        if (tail) atomicOr(out + nw, tail);
       } else {
-        chunk_slow(tb, eplane, splane, c, lane, n, stage, lane_start);
+        chunk_slow(ctl->enc, ks, c, lane, n, image, lane_start);
       }
     }
 
-    // ---- C: exclusive prefix of the tile by decoupled look-back (warp 0)
+    // ---- D: exclusive prefix of the tile by decoupled look-back (warp 0)
     if (warp == 0 && tile > 0) {
       unsigned long long excl = 0;
       long long look = (long long)tile - 1;
@@ -267,22 +361,21 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     __syncthreads();
     if (s_abort) continue;
 
-    // ---- D: write the chunk and its index entry
+    // ---- E: write the chunk and its index entry
     unsigned long long chunk_off = s_tile_base;
     for (uint32_t w = 0; w < warp; ++w) chunk_off += s_chunk_bytes[w];
     if (valid) {
       if (lane == 0) chunk_index[c] = chunk_off;
       uint4* dst4 = reinterpret_cast<uint4*>(payload + chunk_off);
       if (staged) {
-        __syncwarp();
-        const uint4* st4 = reinterpret_cast<const uint4*>(stage);
-        for (uint32_t k = lane; k < chunk_bytes / 16; k += 32) dst4[k] = st4[k];
+        const uint4* im4 = reinterpret_cast<const uint4*>(image);
+        for (uint32_t k = lane; k < chunk_bytes / 16; k += 32) dst4[k] = im4[k];
       } else {
-        // chunk larger than the staging area: OR the bits straight into (zeroed) global memory.
+        // chunk larger than the image area: OR the bits straight into (zeroed) global memory.
         for (uint32_t k = lane; k < chunk_bytes / 16; k += 32) dst4[k] = make_uint4(0, 0, 0, 0);
         __threadfence_block();
         __syncwarp();
-        chunk_slow(tb, eplane, splane, c, lane, n, reinterpret_cast<uint32_t*>(dst4), lane_start);
+        chunk_slow(ctl->enc, ks, c, lane, n, reinterpret_cast<uint32_t*>(dst4), lane_start);
       }
     }
     if (tile == ntiles - 1 && tid == 0) {
@@ -295,10 +388,10 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
 
 }  // namespace
 
-cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* eplane,
-                          const uint32_t* splane, uint64_t n, uint8_t* stream, cudaStream_t cs) {
+cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
+                          const float* cur, uint64_t n, uint8_t* stream, cudaStream_t cs) {
   const WorkspaceLayout W = workspace_layout(n);
-  if (W.ntiles == 0) return cudaSuccess;
+  if (W.nchunks == 0) return cudaSuccess;
   static int blocks_per_sm = 0, sms = 0;
   if (blocks_per_sm == 0) {
     cudaError_t e = cudaFuncSetAttribute(encode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncSmem);
@@ -311,9 +404,10 @@ cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t
     if (e != cudaSuccess) return e;
     blocks_per_sm = bps > 0 ? bps : 1;
   }
+  const uint64_t want = (W.nchunks + kEncWarps - 1) / kEncWarps;
   const uint64_t full = (uint64_t)sms * blocks_per_sm;
-  const unsigned grid = (unsigned)(W.ntiles < full ? W.ntiles : full);
-  encode_kernel<<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, eplane, splane, n, stream);
+  const unsigned grid = (unsigned)(want < full ? want : full);
+  encode_kernel<<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream);
   return cudaGetLastError();
 }
 

@@ -16,10 +16,8 @@ namespace {
 // device context that loads the library, from load to exit.
 constexpr uint64_t kNoAllocMaxN = LC_NOALLOC_MAX_N;
 constexpr uint64_t kNoAllocChunks = (kNoAllocMaxN + kChunkElems - 1) / kChunkElems;
-constexpr uint64_t kNoAllocTiles = (kNoAllocChunks + kEncWarps - 1) / kEncWarps;
 constexpr uint64_t kNoAllocBytes =
-    (sizeof(Control) + 8 * kNoAllocTiles + 255) / 256 * 256 + kNoAllocChunks * kChunkElems +
-    (kNoAllocChunks * (kChunkElems / 8) + 255) / 256 * 256;
+    (sizeof(Control) + 8 * kNoAllocChunks + 255) / 256 * 256 + (kNoAllocChunks * kChunkElems + 255) / 256 * 256;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
@@ -59,14 +57,13 @@ extern "C" int lc_compress_noalloc(const float* base, const float* cur, uint64_t
   uint8_t* w = static_cast<uint8_t*>(scratch);
   Control* ctl = reinterpret_cast<Control*>(w + W.control_off);
   unsigned long long* tiles = reinterpret_cast<unsigned long long*>(w + W.tiles_off);
-  uint8_t* eplane = w + W.eplane_off;
-  uint32_t* splane = reinterpret_cast<uint32_t*>(w + W.splane_off);
+  uint8_t* plane = w + W.plane_off;
 
   // the array keeps what the previous call left: counters, bins and tile descriptors must start at zero
-  if (cudaMemsetAsync(w, 0, W.eplane_off, cs) != cudaSuccess) return LC_ERR_CUDA;
-  if (launch_stats(base, cur, n, ctl, eplane, splane, cs) != cudaSuccess) return LC_ERR_CUDA;
+  if (cudaMemsetAsync(w, 0, W.plane_off, cs) != cudaSuccess) return LC_ERR_CUDA;
+  if (launch_stats(base, cur, n, ctl, plane, cs) != cudaSuccess) return LC_ERR_CUDA;
   if (launch_table(ctl, n, nbits, static_cast<uint8_t*>(stream), cs) != cudaSuccess) return LC_ERR_CUDA;
-  if (launch_encode(ctl, tiles, eplane, splane, n, static_cast<uint8_t*>(stream), cs) != cudaSuccess)
+  if (launch_encode(ctl, tiles, plane, base, cur, n, static_cast<uint8_t*>(stream), cs) != cudaSuccess)
     return LC_ERR_CUDA;
   int32_t status = 0;
   if (cudaMemcpyAsync(&status, &ctl->status, sizeof status, cudaMemcpyDeviceToHost, cs) != cudaSuccess)

@@ -1,10 +1,10 @@
 // Statistics pass: fused delta, (sign, exponent) key extraction, 512-bin histogram with per-bin
-// minimum / maximum, and the 1.125-byte-per-element key plane for the encode pass.
+// minimum / maximum, and the 1-byte-per-element key plane for the encode pass.
 //
 // Paper: Algorithm 1 step 4 (delta against the tracked state) and Section 3.1.1, exponent-based
 // quantization (bucket = identical sign and exponent; representative from the bucket's min and max).
 //
-// Bound: HBM. 8 bytes per element must be read; 1.125 bytes per element are written.
+// Bound: HBM. 8 bytes per element must be read; 1 byte per element is written.
 //
 // Design for a skewed histogram (a handful of exponents hold almost all elements):
 //  * counts live in shared memory as cnt[key][lane]: every lane of a warp owns its own column, so the
@@ -33,6 +33,11 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) {
   return v;
 }
 
+// Top byte = (sign << 7) | (exponent field & 127): bit 31 stays, bits 29..23 move up by one.
+__device__ __forceinline__ uint32_t plane_bits(uint32_t bits) {
+  return ((bits << 1) & 0x7F000000u) | (bits & 0x80000000u);
+}
+
 struct Acc {
   uint32_t* cnt_lane;  // &cnt[lane]
   uint2* mm;
@@ -47,7 +52,7 @@ struct Acc {
 
 __global__ void __launch_bounds__(kStatsThreads, 3)
 stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint64_t n, uint64_t nunits,
-             Control* __restrict__ ctl, uint8_t* __restrict__ eplane, uint32_t* __restrict__ splane) {
+             Control* __restrict__ ctl, uint8_t* __restrict__ plane) {
   extern __shared__ __align__(16) uint32_t smem[];
   uint32_t* cnt = smem;
   uint2* mm = reinterpret_cast<uint2*>(smem + kCntWords);
@@ -62,7 +67,6 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
   for (uint64_t u = warp; u < nunits; u += nwarps) {
     const uint64_t i0 = u * kUnitElems;
     uint32_t ew[kRows];
-    uint32_t signs = 0;
     if (i0 + kUnitElems <= n) {
       const float4* b4 = reinterpret_cast<const float4*>(base + i0) + lane;
       const float4* c4 = reinterpret_cast<const float4*>(cur + i0) + lane;
@@ -82,14 +86,11 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
         acc.add(d1);
         acc.add(d2);
         acc.add(d3);
-        // exponent fields: byte 3 of (bits << 1); gather the four into one word, slot e in byte e.
-        const uint32_t lo = __byte_perm(d0 << 1, d1 << 1, 0x0073);
-        const uint32_t hi = __byte_perm(d2 << 1, d3 << 1, 0x0073);
+        // plane byte = sign, then the low 7 bits of the exponent field: byte 3 of plane_bits(); gather the
+        // four into one word, slot e in byte e.
+        const uint32_t lo = __byte_perm(plane_bits(d0), plane_bits(d1), 0x0073);
+        const uint32_t hi = __byte_perm(plane_bits(d2), plane_bits(d3), 0x0073);
         ew[r] = __byte_perm(lo, hi, 0x5410);
-        signs = __funnelshift_l(d0, signs, 1);
-        signs = __funnelshift_l(d1, signs, 1);
-        signs = __funnelshift_l(d2, signs, 1);
-        signs = __funnelshift_l(d3, signs, 1);
       }
     } else {
       // ragged tail: the last units of the vector, element by element.
@@ -103,16 +104,14 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
             d = __float_as_uint(__fsub_rn(cur[i], base[i]));
             acc.add(d);
           }
-          word |= ((d >> 23) & 255u) << (8 * e);
-          signs = __funnelshift_l(d, signs, 1);
+          word |= (plane_bits(d) >> 24) << (8 * e);
         }
         ew[r] = word;
       }
     }
-    uint4* ep = reinterpret_cast<uint4*>(eplane + i0) + lane;
+    uint4* ep = reinterpret_cast<uint4*>(plane + i0) + lane;
     ep[0] = make_uint4(ew[0], ew[1], ew[2], ew[3]);
     ep[32] = make_uint4(ew[4], ew[5], ew[6], ew[7]);
-    splane[u * 32 + lane] = signs;
   }
   __syncthreads();
 
@@ -131,8 +130,8 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
 
 }  // namespace
 
-cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* eplane,
-                         uint32_t* splane, cudaStream_t cs) {
+cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
+                         cudaStream_t cs) {
   const WorkspaceLayout W = workspace_layout(n);
   if (W.nunits == 0) return cudaSuccess;
   static int blocks_per_sm = 0, sms = 0;
@@ -150,7 +149,7 @@ cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Contro
   const uint64_t want = (W.nunits + kStatsThreads / 32 - 1) / (kStatsThreads / 32);
   const uint64_t full = (uint64_t)sms * blocks_per_sm;
   const unsigned grid = (unsigned)(want < full ? want : full);
-  stats_kernel<<<grid, kStatsThreads, kStatsSmem, cs>>>(base, cur, n, W.nunits, ctl, eplane, splane);
+  stats_kernel<<<grid, kStatsThreads, kStatsSmem, cs>>>(base, cur, n, W.nunits, ctl, plane);
   return cudaGetLastError();
 }
 

@@ -49,6 +49,10 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     return;
   }
 
+  // ---- does the one-byte key plane identify every bucket? (only if all exponent fields are < 128)
+  const bool big = (tid & 255) >= 128 && ctl->count[tid] != 0;
+  const int wide = __syncthreads_or(big);
+
   // ---- priority promotion -------------------------------------------------------------------------
   // thread `tid` < 508 looks at the key of priority position tid: exponent descending, + before -.
   uint32_t key = 0;
@@ -201,6 +205,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   }
   if (tid == 0) {
     ctl->nsym = nsym;
+    ctl->wide = wide ? 1u : 0u;
     ctl->max_len = s_maxlen;
     ctl->payload_bits = s_payload_bits;
     uint8_t* h = stream;

@@ -140,6 +140,32 @@ def test_sweep_distributions(lc, oracle, nbits, dist):
     assert_recover_parity(lc, oracle, base, [got], inplace=(nbits % 2 == 0))
 
 
+def test_large_deltas_bypass_the_key_plane(lc, oracle):
+    # |delta| >= 2 has an exponent field >= 128, which the one-byte key plane cannot hold: the encode
+    # pass then takes its keys from base and cur.
+    from paper_2009_13003_b200 import synth
+
+    n = 300_000 + 77
+    base = synth.normal(n, 1.0, DEV, 31)
+    cur = base + synth.normal(n, 40.0, DEV, 32)
+    got, _ = assert_stream_parity(lc, oracle, base, cur, 5)
+    assert_recover_parity(lc, oracle, base, [got])
+
+
+def test_high_entropy_symbols(lc, oracle):
+    # magnitudes log-uniform over 120 binades, both signs, nbits 8: 255 nearly equiprobable symbols, about
+    # 8 bits per element, so chunks outgrow the default shared-memory areas of both passes.
+    n = 2_000_003
+    g = torch.Generator(device=DEV).manual_seed(33)
+    mag = torch.exp2(torch.rand(n, generator=g, device=DEV) * 120.0 - 124.0)
+    sgn = torch.randint(0, 2, (n,), generator=g, device=DEV) * 2 - 1
+    base = torch.zeros(n, dtype=torch.float32, device=DEV)
+    cur = (mag * sgn).to(torch.float32)
+    got, _ = assert_stream_parity(lc, oracle, base, cur, 8)
+    assert int(np.frombuffer(got[40:48].tobytes(), "<u8")[0]) > 7 * n  # more than 7 bits per element
+    assert_recover_parity(lc, oracle, base, [got, got])
+
+
 def test_deterministic_across_runs(lc):
     base, cur = make_case(5_000_011, 5)
     a, _ = gpu_compress(lc, base, cur, 5)
