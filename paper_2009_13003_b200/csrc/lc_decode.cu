@@ -37,21 +37,20 @@ namespace {
 constexpr int kDecMaxThreads = 512;
 constexpr int kL1Bits = 6;
 constexpr int kL1Rep = 16;
-constexpr int kSubBits = 6;                        // second level: the next 6 bits
-constexpr int kL2Bits = kL1Bits + kSubBits;        // longest code the two table levels resolve
-constexpr int kSubTables = 16;                     // 15 usable + one that only says "longer"
-constexpr uint32_t kSubBytes = (1u << kSubBits) * 8;
+constexpr int kSubBitsMax = 6;                     // second level: the next 6 bits (5 or 4 if many prefixes need one)
+constexpr int kSubBitsMin = 4;
+constexpr int kL2Bits = kL1Bits + kSubBitsMax;     // longest code the two table levels resolve
 constexpr uint32_t kLongCode = 0xFFFFFFFFu;
 constexpr uint32_t kOverrunBytes = 512;  // padding behind the last staging area (see LaneBits::refill)
 static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill guarantee");
 
 // The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory.
 constexpr uint32_t kTableBytes = 8192;
-static_assert((1 << kL1Bits) * kL1Rep * 8 == kTableBytes && kSubTables * kSubBytes == kTableBytes, "table sizes");
+static_assert((1 << kL1Bits) * kL1Rep * 8 == kTableBytes, "table sizes");
 
 struct alignas(16) StreamState {
   uint2* l1;  // [(1 << kL1Bits) * kL1Rep] {bit pattern of rep, code length}; length kLongCode = not resolved here
-  uint2* sub; // [kSubTables][1 << kSubBits] second level: {rep, length} or length kLongCode = longer code
+  uint2* sub; // 8 KB of sub-tables of (1 << sub_bits) entries: {rep, length} or length kLongCode = longer code
   uint32_t sorted_rep[256];           // representatives in canonical (len, id) order
   unsigned long long first_code[64];  // first canonical code of each length
   unsigned long long last_aligned[64]; // largest left-aligned 64-bit window whose code has at most this length
@@ -64,7 +63,8 @@ struct alignas(16) StreamState {
   // validation accumulators
   unsigned long long kraft, count_sum, bit_sum;
   uint32_t seen_max, nused, nsub;
-  uint8_t sub_of_prefix[1 << kL1Bits], prefix_of_sub[kSubTables];
+  uint32_t sub_bits;  // 6, 5 or 4: 16, 32 or 64 sub-tables, the last of which only says "longer"
+  uint8_t sub_of_prefix[1 << kL1Bits], prefix_of_sub[1 << kL1Bits];
 };
 
 static_assert(sizeof(StreamState) % 16 == 0, "the staging areas behind the tables take 16-byte accesses");
@@ -198,20 +198,29 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   __syncthreads();
 
   // ---- lookup tables: canonical decode of each entry's own index
-  // first-level prefixes that belong to longer codes get a sub-table each, as long as there are some left
+  // First-level prefixes that belong to longer codes get a sub-table each. Sub-tables are as deep as
+  // their number allows (8 KB in all, one kept as the table that only says "longer").
   if (tid == 0) {
+    uint32_t misses = 0;
+    if (S.nused >= 2)
+      for (uint32_t idx = 0; idx < (1u << kL1Bits); ++idx) misses += canonical_lookup(S, idx, kL1Bits).y == 0;
+    uint32_t sub_bits = kSubBitsMax;
+    while (sub_bits > kSubBitsMin && misses > (kTableBytes >> (sub_bits + 3)) - 1) sub_bits -= 1;
+    const uint32_t usable = (kTableBytes >> (sub_bits + 3)) - 1;
     uint32_t next = 0;
     for (uint32_t idx = 0; idx < (1u << kL1Bits); ++idx) {
-      uint32_t sub = kSubTables - 1;  // the "longer" sub-table
-      if (S.nused >= 2 && canonical_lookup(S, idx, kL1Bits).y == 0 && next < kSubTables - 1) {
+      uint32_t sub = usable;  // the "longer" sub-table
+      if (S.nused >= 2 && canonical_lookup(S, idx, kL1Bits).y == 0 && next < usable) {
         sub = next++;
         S.prefix_of_sub[sub] = (uint8_t)idx;
       }
       S.sub_of_prefix[idx] = (uint8_t)sub;
     }
     S.nsub = next;
+    S.sub_bits = sub_bits;
   }
   __syncthreads();
+  const uint32_t sub_bits = S.sub_bits;
   for (uint32_t k = tid; k < (1u << kL1Bits) * kL1Rep; k += nthreads) {
     const uint32_t idx = k / kL1Rep;
     uint2 ent;
@@ -220,15 +229,15 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
     } else {
       const uint2 r = canonical_lookup(S, idx, kL1Bits);
       if (r.y) ent = make_uint2(S.sorted_rep[r.x], r.y);
-      else ent = make_uint2(smem_addr(S.sub) + S.sub_of_prefix[idx] * kSubBytes, kLongCode);
+      else ent = make_uint2(smem_addr(S.sub) + ((uint32_t)S.sub_of_prefix[idx] << (sub_bits + 3)), kLongCode);
     }
     S.l1[k] = ent;
   }
-  for (uint32_t k = tid; k < kSubTables << kSubBits; k += nthreads) {
-    const uint32_t sub = k >> kSubBits, j = k & ((1u << kSubBits) - 1);
+  for (uint32_t k = tid; k < kTableBytes / 8; k += nthreads) {
+    const uint32_t sub = k >> sub_bits, j = k & ((1u << sub_bits) - 1);
     uint2 ent = make_uint2(0u, kLongCode);
     if (sub < S.nsub) {
-      const uint2 r = canonical_lookup(S, ((uint32_t)S.prefix_of_sub[sub] << kSubBits) | j, kL2Bits);
+      const uint2 r = canonical_lookup(S, ((uint32_t)S.prefix_of_sub[sub] << sub_bits) | j, kL1Bits + sub_bits);
       if (r.y) ent = make_uint2(S.sorted_rep[r.x], r.y);
     }
     S.sub[k] = ent;
@@ -255,12 +264,12 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 // Two-level table lookup of the code at the top of `hi`: {representative, length}, length kLongCode if
-// the code is longer than kL2Bits. `l1lane` = shared address of this lane's copy of first-level entry 0.
+// the tables do not resolve it. `l1lane` = shared address of this lane's copy of first-level entry 0.
 // The first-level entry of a prefix that belongs to longer codes holds the shared address of the
 // prefix's sub-table, which is read by a predicated load (no branch for the few lanes that need it).
 // Written in PTX so that index scaling and base addition stay multiply-adds (they then run beside the
 // shifts and compares instead of competing with them for the integer pipe).
-__device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane) {
+__device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane, uint32_t sub_shift) {
   uint2 ent;
   asm("{\n\t"
       ".reg .u32 t, a;\n\t"
@@ -275,7 +284,7 @@ __device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane) {
       "@q ld.shared.v2.u32 {%0,%1}, [a];\n\t"
       "}"
       : "=&r"(ent.x), "=&r"(ent.y)
-      : "r"(hi), "r"(l1lane), "n"(32 - kL1Bits), "n"(kL1Rep * 8), "n"(kL1Bits), "n"(32 - kSubBits));
+      : "r"(hi), "r"(l1lane), "n"(32 - kL1Bits), "n"(kL1Rep * 8), "n"(kL1Bits), "r"(sub_shift));
   return ent;
 }
 
@@ -348,7 +357,7 @@ struct LaneBits {
   }
 };
 
-// Code longer than kL2Bits in a staged chunk: canonical search on a 64-bit window read from the
+// Code the tables did not resolve, in a staged chunk: canonical search on a 64-bit window read from the
 // staging area, then re-seat the lane's bit buffer behind the code. Returns the representative.
 __device__ __forceinline__ uint32_t long_code_staged(LaneBits& B, const StreamState& S, const Source& W,
                                                      int32_t* status) {
@@ -357,8 +366,9 @@ __device__ __forceinline__ uint32_t long_code_staged(LaneBits& B, const StreamSt
   const uint32_t w0 = lds_u32(min(at, W.slim)), w1 = lds_u32(min(at + 4u, W.slim)), w2 = lds_u32(min(at + 8u, W.slim));
   const unsigned long long window =
       ((unsigned long long)__funnelshift_l(w1, w0, sh) << 32) | __funnelshift_l(w2, w1, sh);
-  uint32_t L = kL2Bits + 1;
-  while (L < S.max_len && window > S.last_aligned[L]) L += 1;
+  // the first level resolves shorter codes, and so does the prefix's sub-table if it has a real one
+  uint32_t L = kL1Bits + 1 + (S.sub_of_prefix[window >> (64 - kL1Bits)] < S.nsub ? S.sub_bits : 0u);
+  while (L < S.max_len && (S.len_count[L] == 0 || window > S.last_aligned[L])) L += 1;
   const unsigned long long code = window >> (64 - L);
   uint32_t rep = 0;
   if (L <= S.max_len && code >= S.first_code[L] && code - S.first_code[L] < S.len_count[L]) {
@@ -377,11 +387,12 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
                                                     const float* base, float* out, uint64_t c, uint32_t lane,
                                                     int32_t* status) {
   LaneBits bits[KS];
-  uint32_t l1lane[KS];
+  uint32_t l1lane[KS], sub_shift[KS];
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
     bits[s].seek(W[s], start[s]);
     l1lane[s] = smem_addr(S[s].l1) | ((lane & (kL1Rep - 1)) * 8u);
+    sub_shift[s] = 32 - S[s].sub_bits;
   }
   const uint64_t e0 = c * kChunkElems + 4 * lane;
   float4 b = ldg_stream_v4(base + e0);
@@ -401,7 +412,7 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
       uint32_t longest = 0;
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        ent[s] = lookup_code(bits[s].hi, l1lane[s]);
+        ent[s] = lookup_code(bits[s].hi, l1lane[s], sub_shift[s]);
         longest |= ent[s].y;  // lengths are < 64, the marker is all ones
       }
       if (__any_sync(0xffffffffu, longest > 63u)) {
