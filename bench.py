@@ -37,38 +37,74 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def measured_traffic(kernel, n):
+    """DRAM bytes per launch of `kernel` from the committed ncu capture (profiles/traffic.json holds bytes per
+    element measured on a smaller case; every pass is a linear scan, so traffic scales with n). None if absent."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            per_elem = json.load(f)["dram_bytes_per_element"].get(kernel.split("<")[0])
+        return None if per_elem is None else per_elem * n
+    except Exception:
+        return None
+
+
 # ------------------------------------------------------------------------------------------- clocks
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons of one GPU; keeps the samples of the timed region.
+
+    nvidia-smi takes a moment to start, so it is launched before the warm-up; ``mark_start`` and
+    ``stop`` bracket the timed region and only samples that arrived between them are reported.
+    """
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
+        import threading
+
+        self.lines = []  # (arrival time, text)
+        self.t_start = None
         self.proc = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
         except Exception:
             self.proc = None
 
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.perf_counter(), line))
+
+    def wait_ready(self, timeout=10.0):
+        t0 = time.perf_counter()
+        while self.proc is not None and not self.lines and time.perf_counter() - t0 < timeout:
+            time.sleep(0.01)
+
+    def mark_start(self):
+        self.t_start = time.perf_counter()
+
     def stop(self):
+        t_end = time.perf_counter()
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
+        time.sleep(0.03)
         self.proc.terminate()
         try:
-            text, _ = self.proc.communicate(timeout=5)
+            self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-            return out
         sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in text.splitlines():
+        for t, line in list(self.lines):
+            if self.t_start is not None and not (self.t_start <= t <= t_end + 0.02):
+                continue
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 8:
                 continue
@@ -229,16 +265,20 @@ def run_ours(args, rank, world, local_rank):
         lc.compress_async(tracked, u, nbits, sbuf, ws)
         lc.recover_async(u0, streams, out, ws)
 
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
     assert lc.last_status(ws) == 0
+    if sampler:
+        sampler.wait_ready()
 
     # ---- timed region
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     barrier()
     torch.cuda.synchronize()
+    if sampler:
+        sampler.mark_start()
     for k in range(args.steps):
         ev[k][0].record()
         lc.compress_async(tracked, u, nbits, sbuf, ws)
@@ -262,6 +302,18 @@ def run_ours(args, rank, world, local_rank):
     # ---- kernel breakdown of the compress call (events between its kernels; outside the timed region)
     kms = [lc.compress_timed(tracked, u, nbits, sbuf, ws) for _ in range(3)]
     stats_ms, table_ms, encode_ms = (statistics.mean(x[i] for x in kms) for i in range(3))
+
+    # ---- single-stream recovery (the tracked-state update of Algorithm 1 step 7), outside the timed region
+    k1 = []
+    for _ in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        lc.recover_async(u0, streams[:1], out, ws)
+        b.record()
+        torch.cuda.synchronize()
+        k1.append(a.elapsed_time(b))
+    rec1_ms = statistics.median(k1)
+    lc.recover_async(u0, streams, out, ws)  # `out` holds the chain-of-4 result again
 
     # ---- end to end through the host-buffer entry points (pinned host memory, copies inside)
     e2e = None
@@ -296,13 +348,14 @@ def run_ours(args, rank, world, local_rank):
     sbar = [b / n for b in stream_bytes]
     kernels = {
         "stats_kernel": {"ms": stats_ms, "alg_bytes": 8.0 * n},
-        "encode_kernel": {"ms": encode_ms, "alg_bytes": stream_bytes[-1] + 1.125 * n},
+        "encode_kernel": {"ms": encode_ms, "alg_bytes": stream_bytes[-1] + 1.0 * n},
         "decode_kernel<%d>" % min(chain, 4): {"ms": rec, "alg_bytes": 8.0 * n + sum(stream_bytes)},
     }
     dom = max(kernels, key=lambda k: kernels[k]["ms"])
     achieved = kernels[dom]["alg_bytes"] / (kernels[dom]["ms"] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": peak_kind + " (STREAM-style copy)", "traffic": None,
+                "frac": achieved / peak, "peak_source": peak_kind + " (STREAM-style copy)",
+                "traffic": measured_traffic(dom, n),
                 "per_kernel": {k: {"ms": v["ms"], "achieved_gbs": v["alg_bytes"] / (v["ms"] * 1e-3) / 1e9,
                                    "frac": v["alg_bytes"] / (v["ms"] * 1e-3) / 1e9 / peak}
                                for k, v in kernels.items()}}
@@ -320,6 +373,8 @@ def run_ours(args, rank, world, local_rank):
                      "kernels_ms": {"stats": stats_ms, "table": table_ms, "encode": encode_ms}},
         "recover": {"ms": rec, "state_gbs": 4 * n / (rec * 1e-3) / 1e9, "alg_gbs": rec_alg,
                     "frac_of_peak": rec_alg / peak},
+        "recover_k1": {"ms": rec1_ms, "alg_gbs": (8.0 * n + stream_bytes[0]) / (rec1_ms * 1e-3) / 1e9,
+                       "frac_of_peak": (8.0 * n + stream_bytes[0]) / (rec1_ms * 1e-3) / 1e9 / peak},
         "ratio": {"stream": 4.0 * n / stream_bytes[-1], "bits_per_element": 8.0 * sbar[-1]},
         "roofline": roofline, "clocks": clocks, "e2e": e2e,
         "gpu_launches": 4 * args.steps,  # stats, table, encode, decode per step
@@ -332,7 +387,7 @@ def run_ours(args, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=60)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--elems", type=int, default=0, help="override the element count (profiling on small cases)")

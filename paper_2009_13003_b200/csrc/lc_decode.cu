@@ -577,23 +577,43 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
     sms = v;
   }
   const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
-  // One CTA per SM. Staging per warp and stream: 1.03 x the largest average chunk of the streams (from
-  // the buffer sizes, which bound the payload), with as many warps (16, 12 or 8) as then fit.
+  // Staging per warp and stream: 1.03 x the largest average chunk of the streams (from the buffer sizes,
+  // which bound the payload). Among CTAs of 16, 12 and 8 warps, take the shape that puts most warps on an
+  // SM (shared memory and registers both count; with four streams that is one CTA of 16 warps, with one
+  // stream several smaller CTAs).
   uint64_t avg = 0;
   for (int s = 0; s < KS; ++s) {
     const uint64_t index_bytes = 72 * nchunks;  // lane and chunk index entries are not staged
     const uint64_t a = (streams.bytes[s] > index_bytes ? streams.bytes[s] - index_bytes : 0) / (nchunks ? nchunks : 1);
     avg = a > avg ? a : avg;
   }
-  const uint64_t want_stage = align_up(avg + avg / 32 + 48, 16);
-  uint32_t warps = 16;
-  while (warps > 8 && kTables + (uint64_t)warps * KS * want_stage > kMaxDyn) warps -= 4;
-  uint32_t stage = ((kMaxDyn - kTables) / (warps * KS)) / 16 * 16;
-  if (stage > kChunkElems * 8 + 16) stage = kChunkElems * 8 + 16;
-  const uint32_t dyn = kTables + warps * KS * stage + kOverrunBytes;
+  uint64_t want_stage = align_up(avg + avg / 32 + 48, 16);
+  if (want_stage > kChunkElems * 8 + 16) want_stage = kChunkElems * 8 + 16;
+  uint32_t warps = 8, stage = 0, dyn = 0, best_warps_per_sm = 0, ctas_per_sm = 1;
+  for (uint32_t w = 16; w >= 8; w -= 4) {
+    uint32_t st = (uint32_t)want_stage;
+    if (kTables + (uint64_t)w * KS * st > kMaxDyn) {
+      if (w > 8) continue;                               // try fewer warps first
+      st = ((kMaxDyn - kTables) / (w * KS)) / 16 * 16;   // last resort: what fits; large chunks decode from global
+    }
+    const uint32_t d = kTables + w * KS * st + kOverrunBytes;
+    int bps = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, decode_kernel<KS>, (int)(w * 32), d) != cudaSuccess)
+      return cudaErrorUnknown;
+    if (bps < 1) continue;
+    if ((uint32_t)bps * w > best_warps_per_sm) {
+      best_warps_per_sm = (uint32_t)bps * w;
+      warps = w;
+      stage = st;
+      dyn = d;
+      ctas_per_sm = (uint32_t)bps;
+    }
+  }
+  if (best_warps_per_sm == 0) return cudaErrorLaunchOutOfResources;
   uint64_t want = (nchunks + warps - 1) / warps;
   if (want == 0) want = 1;  // still validates the streams
-  const unsigned grid = (unsigned)(want < (uint64_t)sms ? want : (uint64_t)sms);
+  const uint64_t full = (uint64_t)sms * ctas_per_sm;
+  const unsigned grid = (unsigned)(want < full ? want : full);
   decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, stage);
   return cudaGetLastError();
 }
