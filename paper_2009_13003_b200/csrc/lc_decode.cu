@@ -65,6 +65,9 @@ struct alignas(16) StreamState {
   uint32_t seen_max, nused, nsub;
   uint32_t sub_bits;  // 6, 5 or 4: 16, 32 or 64 sub-tables, the last of which only says "longer"
   uint8_t sub_of_prefix[1 << kL1Bits], prefix_of_sub[1 << kL1Bits];
+  uint8_t sym_len[256];   // code length by symbol id
+  uint32_t miss_count[2];  // first-level prefixes without a short code, per warp of 32 prefixes
+  alignas(16) uint8_t hdr[kHeaderBytes];  // the stream header, staged
 };
 
 static_assert(sizeof(StreamState) % 16 == 0, "the staging areas behind the tables take 16-byte accesses");
@@ -93,27 +96,31 @@ __device__ __forceinline__ uint2 canonical_lookup(const StreamState& S, uint32_t
 __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8_t* __restrict__ s,
                               uint64_t bytes, uint64_t n, int* s_err) {
   const int tid = threadIdx.x, nthreads = blockDim.x;
+  if (tid < 4 && bytes >= kHeaderBytes)
+    reinterpret_cast<uint4*>(S.hdr)[tid] = __ldg(reinterpret_cast<const uint4*>(s) + tid);
+  __syncthreads();
   if (tid == 0) {
     int err = 0;
+    const uint8_t* h = S.hdr;
     S.l1 = reinterpret_cast<uint2*>(tables);
     S.sub = reinterpret_cast<uint2*>(tables + kTableBytes);
     S.kraft = 0; S.count_sum = 0; S.bit_sum = 0; S.seen_max = 0; S.nused = 0; S.only_rep = 0;
     if (bytes < kHeaderBytes) {
       err = LC_ERR_FORMAT;
     } else {
-      const uint32_t nbits = s[6];
-      S.n = load_le(s + 8, 8);
-      S.nsym = (uint32_t)load_le(s + 16, 4);
-      S.max_len = (uint32_t)load_le(s + 20, 4);
-      S.nchunks = (uint32_t)load_le(s + 32, 4);
-      S.payload_bits = load_le(s + 40, 8);
-      S.total_bytes = load_le(s + 48, 8);
-      S.payload_off = load_le(s + 56, 8);
-      const bool magic = s[0] == 'L' && s[1] == 'C' && s[2] == 'C' && s[3] == '1';
-      if (!magic || load_le(s + 4, 2) != 1 || nbits < 1 || nbits > 8 || s[7] != 0) err = LC_ERR_FORMAT;
+      const uint32_t nbits = h[6];
+      S.n = load_le(h + 8, 8);
+      S.nsym = (uint32_t)load_le(h + 16, 4);
+      S.max_len = (uint32_t)load_le(h + 20, 4);
+      S.nchunks = (uint32_t)load_le(h + 32, 4);
+      S.payload_bits = load_le(h + 40, 8);
+      S.total_bytes = load_le(h + 48, 8);
+      S.payload_off = load_le(h + 56, 8);
+      const bool magic = h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1';
+      if (!magic || load_le(h + 4, 2) != 1 || nbits < 1 || nbits > 8 || h[7] != 0) err = LC_ERR_FORMAT;
       else if (S.nsym < 1 || S.nsym > (1u << nbits) || S.max_len > 63) err = LC_ERR_FORMAT;
-      else if (load_le(s + 24, 4) != kChunkElems || load_le(s + 28, 2) != kLanes ||
-               load_le(s + 30, 2) != kGroup || load_le(s + 36, 4) != kPayloadAlign) err = LC_ERR_FORMAT;
+      else if (load_le(h + 24, 4) != kChunkElems || load_le(h + 28, 2) != kLanes ||
+               load_le(h + 30, 2) != kGroup || load_le(h + 36, 4) != kPayloadAlign) err = LC_ERR_FORMAT;
       else if (S.n != n) err = S.n < (1ull << 32) ? LC_ERR_MISMATCH : LC_ERR_FORMAT;
       if (!err) {
         const StreamLayout L = stream_layout(S.n, S.nsym);
@@ -142,11 +149,12 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   unsigned long long my_count = 0;
   bool entry_bad = false;
   if (tid < (int)nsym) {
-    const uint8_t* e = s + kHeaderBytes + kTableEntryBytes * tid;
-    my_len = e[2];
-    my_rep = (uint32_t)load_le(e + 4, 4);
-    my_count = load_le(e + 8, 8);
-    entry_bad = e[3] != 0 || my_len > 63 || (my_count == 0 && my_len != 0);
+    const uint4 e = __ldg(reinterpret_cast<const uint4*>(s + kHeaderBytes) + tid);  // key:16 len:8 pad:8 | rep | count
+    my_len = (e.x >> 16) & 255u;
+    my_rep = e.y;
+    my_count = ((unsigned long long)e.w << 32) | e.z;
+    entry_bad = (e.x >> 24) != 0 || my_len > 63 || (my_count == 0 && my_len != 0);
+    S.sym_len[tid] = (uint8_t)my_len;
     if (my_count != 0) {
       atomicAdd(&S.count_sum, my_count);
       atomicAdd(&S.bit_sum, my_count * my_len);
@@ -191,7 +199,7 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   if (S.nused >= 2 && tid < (int)nsym && my_count != 0) {
     // rank among the symbols of the same length with smaller id (zero-count symbols have length 0)
     uint32_t r = 0;
-    for (int j = 0; j < tid; ++j) r += (s[kHeaderBytes + kTableEntryBytes * j + 2] == my_len) ? 1u : 0u;
+    for (int j = 0; j < tid; ++j) r += (S.sym_len[j] == my_len) ? 1u : 0u;
     S.sorted_rep[S.len_offset[my_len] + r] = my_rep;
   }
   if (S.nused < 2 && tid == 0) S.sorted_rep[0] = S.only_rep;
@@ -200,24 +208,28 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   // ---- lookup tables: canonical decode of each entry's own index
   // First-level prefixes that belong to longer codes get a sub-table each. Sub-tables are as deep as
   // their number allows (8 KB in all, one kept as the table that only says "longer").
-  if (tid == 0) {
-    uint32_t misses = 0;
-    if (S.nused >= 2)
-      for (uint32_t idx = 0; idx < (1u << kL1Bits); ++idx) misses += canonical_lookup(S, idx, kL1Bits).y == 0;
-    uint32_t sub_bits = kSubBitsMax;
-    while (sub_bits > kSubBitsMin && misses > (kTableBytes >> (sub_bits + 3)) - 1) sub_bits -= 1;
-    const uint32_t usable = (kTableBytes >> (sub_bits + 3)) - 1;
-    uint32_t next = 0;
-    for (uint32_t idx = 0; idx < (1u << kL1Bits); ++idx) {
+  {
+    const bool miss = tid < (1 << kL1Bits) && S.nused >= 2 && canonical_lookup(S, tid, kL1Bits).y == 0;
+    const uint32_t ballot = __ballot_sync(0xffffffffu, miss);
+    if (tid < (1 << kL1Bits) && (tid & 31) == 0) S.miss_count[tid >> 5] = __popc(ballot);
+    __syncthreads();
+    if (tid < (1 << kL1Bits)) {
+      const uint32_t misses = S.miss_count[0] + S.miss_count[1];
+      uint32_t sub_bits = kSubBitsMax;
+      while (sub_bits > kSubBitsMin && misses > (kTableBytes >> (sub_bits + 3)) - 1) sub_bits -= 1;
+      const uint32_t usable = (kTableBytes >> (sub_bits + 3)) - 1;
+      const uint32_t rank = __popc(ballot & ((1u << (tid & 31)) - 1)) + (tid >= 32 ? S.miss_count[0] : 0u);
       uint32_t sub = usable;  // the "longer" sub-table
-      if (S.nused >= 2 && canonical_lookup(S, idx, kL1Bits).y == 0 && next < usable) {
-        sub = next++;
-        S.prefix_of_sub[sub] = (uint8_t)idx;
+      if (miss && rank < usable) {
+        sub = rank;
+        S.prefix_of_sub[sub] = (uint8_t)tid;
       }
-      S.sub_of_prefix[idx] = (uint8_t)sub;
+      S.sub_of_prefix[tid] = (uint8_t)sub;
+      if (tid == 0) {
+        S.nsub = misses < usable ? misses : usable;
+        S.sub_bits = sub_bits;
+      }
     }
-    S.nsub = next;
-    S.sub_bits = sub_bits;
   }
   __syncthreads();
   const uint32_t sub_bits = S.sub_bits;
