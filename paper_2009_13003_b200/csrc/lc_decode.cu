@@ -327,40 +327,71 @@ __device__ __noinline__ uint2 decode_any(const StreamState& S, const uint32_t* g
   return make_uint2(0u, S.max_len);
 }
 
-// A lane's read state in one stream of a staged chunk: `cnt` valid bits at the top of hi:lo (the bits
-// below are zero); `next` = shared address of the next word to load.
+// A lane's read state in one stream: `cnt` valid bits at the top of hi:lo (the bits below are zero).
+// STAGED: the chunk's words are in the warp's staging area and `next` is the shared address of the next
+// word to load. Otherwise (a chunk too large to stage) they are read from global memory and `next` is a
+// word index.
+template <bool STAGED>
 struct LaneBits {
   uint32_t hi, lo;
   int cnt;
   uint32_t next;
 
-  __device__ __forceinline__ uint32_t bitpos(const Source& W) const { return (next - W.sbase) * 8u - (uint32_t)cnt; }
+  // word `idx` of the chunk, 0 beyond its end
+  __device__ __forceinline__ static uint32_t word(const Source& W, uint32_t idx) {
+    if (STAGED) return lds_u32(min(W.sbase + idx * 4u, W.slim));
+    return idx < W.nw ? __ldg(W.g + idx) : 0u;
+  }
+  __device__ __forceinline__ uint32_t bitpos(const Source& W) const {
+    return (STAGED ? (next - W.sbase) * 8u : next * 32u) - (uint32_t)cnt;
+  }
   __device__ __forceinline__ void seek(const Source& W, uint32_t pos) {
-    const uint32_t at = W.sbase + (pos >> 5) * 4u, sh = pos & 31;
-    const uint32_t w0 = lds_u32(min(at, W.slim)), w1 = lds_u32(min(at + 4u, W.slim));
+    const uint32_t idx = pos >> 5, sh = pos & 31;
+    const uint32_t w0 = word(W, idx), w1 = word(W, idx + 1);
     hi = __funnelshift_l(w1, w0, sh);
     lo = w1 << sh;
     cnt = 64 - (int)sh;
-    next = min(at + 8u, W.slim);
+    next = STAGED ? min(W.sbase + (idx + 2) * 4u, W.slim) : idx + 2;
   }
   // Tops the buffer up with one word if 32 bits or fewer are left; afterwards cnt >= 33. All predicated.
-  // The load is not clamped: between two seeks (which do clamp) `next` moves by at most 64 words, and the
-  // kernel's shared memory ends with kOverrunBytes of padding, so a damaged stream can make a lane read
-  // stale shared memory but never leave the allocation.
-  __device__ __forceinline__ void refill() {
-    asm volatile(
-        "{\n\t"
-        ".reg .pred q;\n\t"
-        ".reg .u32 w, t;\n\t"
-        "setp.le.s32 q, %2, 32;\n\t"
-        "@q ld.shared.u32 w, [%3];\n\t"
-        "@q shf.r.clamp.b32 t, w, 0, %2;\n\t"   // high word of (w:0) >> cnt, i.e. w >> cnt (0 when cnt == 32)
-        "@q or.b32 %0, %0, t;\n\t"
-        "@q shf.r.clamp.b32 %1, 0, w, %2;\n\t"  // low word of (w:0) >> cnt; lo was 0 because cnt <= 32
-        "@q add.s32 %2, %2, 32;\n\t"
-        "@q add.u32 %3, %3, 4;\n\t"
-        "}"
-        : "+r"(hi), "+r"(lo), "+r"(cnt), "+r"(next));
+  // STAGED: the load is not clamped: between two seeks (which do clamp) `next` moves by at most 64 words,
+  // and the kernel's shared memory ends with kOverrunBytes of padding, so a damaged stream can make a lane
+  // read stale shared memory but never leave the allocation.
+  __device__ __forceinline__ void refill(const Source& W) {
+    if (STAGED) {
+      asm volatile(
+          "{\n\t"
+          ".reg .pred q;\n\t"
+          ".reg .u32 w, t;\n\t"
+          "setp.le.s32 q, %2, 32;\n\t"
+          "@q ld.shared.u32 w, [%3];\n\t"
+          "@q shf.r.clamp.b32 t, w, 0, %2;\n\t"   // high word of (w:0) >> cnt, i.e. w >> cnt (0 when cnt == 32)
+          "@q or.b32 %0, %0, t;\n\t"
+          "@q shf.r.clamp.b32 %1, 0, w, %2;\n\t"  // low word of (w:0) >> cnt; lo was 0 because cnt <= 32
+          "@q add.s32 %2, %2, 32;\n\t"
+          "@q add.u32 %3, %3, 4;\n\t"
+          "}"
+          : "+r"(hi), "+r"(lo), "+r"(cnt), "+r"(next));
+    } else {
+      asm volatile(
+          "{\n\t"
+          ".reg .pred q, r;\n\t"
+          ".reg .u32 w, t;\n\t"
+          ".reg .u64 a;\n\t"
+          "setp.le.s32 q, %2, 32;\n\t"
+          "setp.lt.and.u32 r, %3, %5, q;\n\t"     // words beyond the chunk read as 0
+          "mov.u32 w, 0;\n\t"
+          "mad.wide.u32 a, %3, 4, %4;\n\t"
+          "@r ld.global.nc.u32 w, [a];\n\t"
+          "@q shf.r.clamp.b32 t, w, 0, %2;\n\t"
+          "@q or.b32 %0, %0, t;\n\t"
+          "@q shf.r.clamp.b32 %1, 0, w, %2;\n\t"
+          "@q add.s32 %2, %2, 32;\n\t"
+          "@q add.u32 %3, %3, 1;\n\t"
+          "}"
+          : "+r"(hi), "+r"(lo), "+r"(cnt), "+r"(next)
+          : "l"(W.g), "r"(W.nw));
+    }
   }
   __device__ __forceinline__ void consume(uint32_t len) {
     hi = __funnelshift_l(lo, hi, len);
@@ -369,13 +400,14 @@ struct LaneBits {
   }
 };
 
-// Code the tables did not resolve, in a staged chunk: canonical search on a 64-bit window read from the
-// staging area, then re-seat the lane's bit buffer behind the code. Returns the representative.
-__device__ __forceinline__ uint32_t long_code_staged(LaneBits& B, const StreamState& S, const Source& W,
-                                                     int32_t* status) {
+// Code the tables did not resolve: canonical search on a 64-bit window read from the chunk, then re-seat
+// the lane's bit buffer behind the code. Returns the representative.
+template <bool STAGED>
+__device__ __forceinline__ uint32_t long_code(LaneBits<STAGED>& B, const StreamState& S, const Source& W,
+                                              int32_t* status) {
   const uint32_t pos = B.bitpos(W);
-  const uint32_t at = W.sbase + (pos >> 5) * 4u, sh = pos & 31;
-  const uint32_t w0 = lds_u32(min(at, W.slim)), w1 = lds_u32(min(at + 4u, W.slim)), w2 = lds_u32(min(at + 8u, W.slim));
+  const uint32_t idx = pos >> 5, sh = pos & 31;
+  const uint32_t w0 = B.word(W, idx), w1 = B.word(W, idx + 1), w2 = B.word(W, idx + 2);
   const unsigned long long window =
       ((unsigned long long)__funnelshift_l(w1, w0, sh) << 32) | __funnelshift_l(w2, w1, sh);
   // the first level resolves shorter codes, and so does the prefix's sub-table if it has a real one
@@ -392,13 +424,13 @@ __device__ __forceinline__ uint32_t long_code_staged(LaneBits& B, const StreamSt
   return rep;
 }
 
-// Full chunk, every stream staged: the hot loop. Per step a lane decodes 4 elements x KS streams; the
-// KS streams are independent dependency chains and are written interleaved.
-template <int KS>
-__device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const Source* W, const uint32_t* start,
+// Full chunk: the hot loop. Per step a lane decodes 4 elements x KS streams; the KS streams are
+// independent dependency chains and are written interleaved.
+template <int KS, bool STAGED>
+__device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const Source* W, const uint32_t* start,
                                                     const float* base, float* out, uint64_t c, uint32_t lane,
                                                     int32_t* status) {
-  LaneBits bits[KS];
+  LaneBits<STAGED> bits[KS];
   uint32_t l1lane[KS], sub_shift[KS];
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
@@ -418,7 +450,7 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
     for (int e = 0; e < 4; ++e) {
       if ((e & 1) == 0) {
 #pragma unroll
-        for (int s = 0; s < KS; ++s) bits[s].refill();
+        for (int s = 0; s < KS; ++s) bits[s].refill(W[s]);
       }
       uint2 ent[KS];
       uint32_t longest = 0;
@@ -430,7 +462,7 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
       if (__any_sync(0xffffffffu, longest > 63u)) {
 #pragma unroll
         for (int s = 0; s < KS; ++s) {
-          if (ent[s].y > 63u) ent[s] = make_uint2(long_code_staged(bits[s], S[s], W[s], status), 0u);  // consumed
+          if (ent[s].y > 63u) ent[s] = make_uint2(long_code<STAGED>(bits[s], S[s], W[s], status), 0u);  // consumed
         }
       }
 #pragma unroll
@@ -444,7 +476,7 @@ __device__ __forceinline__ void decode_chunk_staged(const StreamState* S, const 
 }
 static_assert(kL1Rep * 8 == 128, "first-level entries of one index span 128 bytes");
 
-// Any chunk (ragged, or too large to stage), read from global memory; plain code, no warp votes.
+// The ragged last chunk, read from global memory; plain code, no warp votes.
 struct GlobalChunk {
   const uint32_t* g[4];
   uint32_t nw[4];
@@ -556,8 +588,10 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
     }
     cp_async_wait_all();
     __syncwarp();
-    if (fits && (c + 1) * kChunkElems <= n) decode_chunk_staged<KS>(S, W, start, base, out, c, lane, status);
-    else {
+    if ((c + 1) * kChunkElems <= n) {
+      if (fits) decode_chunk_fast<KS, true>(S, W, start, base, out, c, lane, status);
+      else decode_chunk_fast<KS, false>(S, W, start, base, out, c, lane, status);
+    } else {
       GlobalChunk G;
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
@@ -622,6 +656,22 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
     }
   }
   if (best_warps_per_sm == 0) return cudaErrorLaunchOutOfResources;
+  // chunk sizes vary around the average: give the staging areas whatever shared memory this shape leaves
+  {
+    const uint32_t budget = kSmemPerSm / ctas_per_sm - 1024 - 64;
+    if (budget > kTables + kOverrunBytes) {
+      uint32_t st = ((budget - kTables - kOverrunBytes) / (warps * KS)) / 16 * 16;
+      if (st > kChunkElems * 8 + 16) st = kChunkElems * 8 + 16;
+      const uint32_t d = kTables + warps * KS * st + kOverrunBytes;
+      int bps = 0;
+      if (st > stage && d <= kMaxDyn + kOverrunBytes &&
+          cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, decode_kernel<KS>, (int)(warps * 32), d) == cudaSuccess &&
+          (uint32_t)bps >= ctas_per_sm) {
+        stage = st;
+        dyn = d;
+      }
+    }
+  }
   uint64_t want = (nchunks + warps - 1) / warps;
   if (want == 0) want = 1;  // still validates the streams
   const uint64_t full = (uint64_t)sms * ctas_per_sm;
