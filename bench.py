@@ -38,12 +38,13 @@ def measured_peak():
 
 
 def measured_traffic(kernel, n):
-    """DRAM bytes per launch of `kernel` from the committed ncu capture (profiles/traffic.json holds bytes per
+    """DRAM bytes per launch of `kernel` from the committed ncu capture (profiles/traffic.txt holds bytes per
     element measured on a smaller case; every pass is a linear scan, so traffic scales with n). None if absent."""
     try:
-        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
-            per_elem = json.load(f)["dram_bytes_per_element"].get(kernel.split("<")[0])
-        return None if per_elem is None else per_elem * n
+        with open(os.path.join(ROOT, "profiles", "traffic.txt")) as f:
+            table = dict(line.split() for line in f if line.strip() and not line.startswith("#"))
+        per_elem = table.get(kernel.split("<")[0])
+        return None if per_elem is None else float(per_elem) * n
     except Exception:
         return None
 
