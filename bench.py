@@ -178,7 +178,11 @@ def run_reference(args, rank):
     from paper_2009_13003_b200 import synth
 
     cfg = synth.CONFIGS[WORKLOAD]
-    m = CPU_SAMPLE_ELEMS
+    # bounded sample: the oracle does about 12 M elements per second of (compress + chain-of-4 recover) on one
+    # core, and the whole run (set-up, warm-up, steps) should end within a few minutes
+    budget_s = 150.0
+    m = int(budget_s / (args.steps + args.warmup + 2) * 12e6) // 4096 * 4096
+    m = max(4096, min(CPU_SAMPLE_ELEMS, m, cfg.n))
     u0 = synth.base_state(cfg, "cpu", m).numpy()
     tracked, u, streams = u0.copy(), u0.copy(), []
     for t in range(1, cfg.chain + 1):
