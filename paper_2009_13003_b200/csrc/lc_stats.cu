@@ -41,12 +41,32 @@ __device__ __forceinline__ uint32_t plane_bits(uint32_t bits) {
 struct Acc {
   uint32_t* cnt_lane;  // &cnt[lane]
   uint2* mm;
+  __device__ __forceinline__ void improve(uint32_t bits, uint32_t key, uint2 cur) {
+    if (~bits > cur.x) atomicMax(&mm[key].x, ~bits);
+    if (bits > cur.y) atomicMax(&mm[key].y, bits);
+  }
   __device__ __forceinline__ void add(uint32_t bits) {
     const uint32_t key = bits >> 23;
     atomicAdd(cnt_lane + key * 32, 1u);
-    const uint2 cur = mm[key];
-    if (~bits > cur.x) atomicMax(&mm[key].x, ~bits);
-    if (bits > cur.y) atomicMax(&mm[key].y, bits);
+    improve(bits, key, mm[key]);
+  }
+  // Four elements at once: the four reads of the running min / max pairs go out together, and one test
+  // covers all eight comparisons, because after the first few elements none of them ever holds.
+  __device__ __forceinline__ void add4(uint32_t d0, uint32_t d1, uint32_t d2, uint32_t d3) {
+    const uint32_t k0 = d0 >> 23, k1 = d1 >> 23, k2 = d2 >> 23, k3 = d3 >> 23;
+    const uint2 c0 = mm[k0], c1 = mm[k1], c2 = mm[k2], c3 = mm[k3];
+    atomicAdd(cnt_lane + k0 * 32, 1u);
+    atomicAdd(cnt_lane + k1 * 32, 1u);
+    atomicAdd(cnt_lane + k2 * 32, 1u);
+    atomicAdd(cnt_lane + k3 * 32, 1u);
+    const bool any = (~d0 > c0.x) | (d0 > c0.y) | (~d1 > c1.x) | (d1 > c1.y) | (~d2 > c2.x) | (d2 > c2.y) |
+                     (~d3 > c3.x) | (d3 > c3.y);
+    if (any) {
+      improve(d0, k0, c0);
+      improve(d1, k1, c1);
+      improve(d2, k2, c2);
+      improve(d3, k3, c3);
+    }
   }
 };
 
@@ -82,10 +102,7 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
         const uint32_t d1 = __float_as_uint(__fsub_rn(c[r].y, b[r].y));
         const uint32_t d2 = __float_as_uint(__fsub_rn(c[r].z, b[r].z));
         const uint32_t d3 = __float_as_uint(__fsub_rn(c[r].w, b[r].w));
-        acc.add(d0);
-        acc.add(d1);
-        acc.add(d2);
-        acc.add(d3);
+        acc.add4(d0, d1, d2, d3);
         // plane byte = sign, then the low 7 bits of the exponent field: byte 3 of plane_bits(); gather the
         // four into one word, slot e in byte e.
         const uint32_t lo = __byte_perm(plane_bits(d0), plane_bits(d1), 0x0073);
