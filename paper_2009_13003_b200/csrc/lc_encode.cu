@@ -8,8 +8,9 @@
 //   A. every lane codes its 128 elements into its own column of a warp-private word matrix in shared
 //      memory (word k of lane t at k*32 + t: plain stores, no bank conflicts, no atomics). Code and
 //      length come packed in one 32-bit table entry (a 16-byte entry made the lookups saturate the
-//      shared-memory pipe); the rare codes of 27..32 bits are fetched by a predicated second load.
-//      Emitting a finished word is a handful of predicated instructions;
+//      shared-memory pipe) and two neighbouring codes are appended as one; the rare codes of 17..32 bits
+//      sit behind one vote per four elements. Emitting a finished word is a handful of predicated
+//      instructions;
 //   B. a warp shuffle scan of the lane bit counts gives every lane its bit offset in the chunk (the
 //      lane index of the stream) and the chunk its size, which is published at once;
 //   C. the lanes' words are shifted to their bit offsets and ORed into the chunk image (shared memory);
@@ -40,10 +41,11 @@ constexpr uint32_t kSpinLimit = 1u << 20;
 
 constexpr uint32_t kPackedLenShift = 26;                      // packed entry: length << 26 | code
 constexpr uint32_t kPackedCodeMask = (1u << kPackedLenShift) - 1;
+constexpr uint32_t kPackedMaxLen = 16;                        // two packed codes make one append of <= 32 bits
 constexpr uint32_t kPackedLong = 63;                          // length field of a code that does not fit
 
 struct Tables {
-  uint32_t packed[256];  // by plane byte: length << 26 | code for codes of up to 26 bits, else length field 63
+  uint32_t packed[256];  // by plane byte: length << 26 | code for codes of up to 16 bits, else length field 63
   uint2 full[256];       // by plane byte: {code, length} for codes of up to 32 bits
 };
 
@@ -164,7 +166,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
   for (uint32_t b = tid; b < 256; b += kEncThreads) {
     const EncEntry e = ctl->enc[((b & 128u) << 1) | (b & 127u)];
     tb.full[b] = make_uint2(e.code_lo, e.len);
-    tb.packed[b] = e.len <= kPackedLenShift ? (e.len << kPackedLenShift) | e.code_lo : kPackedLong << kPackedLenShift;
+    tb.packed[b] = e.len <= kPackedMaxLen ? (e.len << kPackedLenShift) | e.code_lo : kPackedLong << kPackedLenShift;
   }
   __syncthreads();
 
@@ -196,27 +198,25 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
       asm volatile("ld.shared.u32 %0, [%1];" : "=r"(g[e]) : "r"(packed_addr + b * 4u));
     }
   };
-  // Appends the four codes of `word`, whose packed entries are g. Only the marker has bit 31 set (packed
-  // lengths are <= 26), so one test per row finds the rare codes of 27..32 bits, which come from `full`.
+  // Appends the four codes of `word`, whose packed entries are g. Packed codes have at most 16 bits, so two
+  // neighbours are joined into one append of at most 32 bits (half the accumulator and flush work). Only the
+  // marker has bit 31 set, so one test per row finds the rare longer codes; that row then appends its four
+  // codes one by one from `full`.
   auto put4 = [&](ColumnPacker& pk, uint32_t word, const uint32_t (&g)[4]) {
-    uint32_t code[4], len[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      len[e] = g[e] >> kPackedLenShift;
-      code[e] = g[e] & kPackedCodeMask;
-    }
     if (__any_sync(0xffffffffu, (int)(g[0] | g[1] | g[2] | g[3]) < 0)) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        if ((int)g[e] < 0) {
-          const uint2 f = tb.full[__byte_perm(word, 0u, 0x4440 + e)];
-          code[e] = f.x;
-          len[e] = f.y;
-        }
+        const uint2 f = tb.full[__byte_perm(word, 0u, 0x4440 + e)];
+        pk.put(f.x, f.y);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; e += 2) {
+        const uint32_t l0 = g[e] >> kPackedLenShift, l1 = g[e + 1] >> kPackedLenShift;
+        const uint32_t c0 = g[e] & kPackedCodeMask, c1 = g[e + 1] & kPackedCodeMask;
+        pk.put((c0 << l1) | c1, l0 + l1);
       }
     }
-#pragma unroll
-    for (int e = 0; e < 4; ++e) pk.put(code[e], len[e]);
   };
   auto fast_chunk = [&](uint64_t cc) { return cc < nchunks && (cc + 1) * kChunkElems <= n && !long_codes && !ks.wide; };
 
