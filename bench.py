@@ -271,6 +271,15 @@ def run_ours(args, rank, world, local_rank):
     out = torch.empty_like(u0)
     stream_bytes = [int(s.numel()) for s in streams]
     torch.cuda.synchronize()
+    # size of the last snapshot under the paper's three stages (Section 4.3: E, E+P, E+P+H), as fractions of
+    # the full fp32 state; the first two by the paper's size model n*ceil(log2 k) + k*32 bits
+    count, _, _ = lc.debug_bins(ws)
+    k_e = int((count > 0).sum())
+    nsym = int(lc.stream_info(streams[-1]).nsym)
+    width = lambda k: max(1, (k - 1).bit_length())
+    size_model = {"occupied_buckets": k_e, "kept_symbols": nsym,
+                  "E": (n * width(k_e) + 32 * k_e) / (32.0 * n), "E+P": (n * width(nsym) + 32 * nsym) / (32.0 * n),
+                  "E+P+H": 8.0 * stream_bytes[-1] / (32.0 * n)}
 
     def step():
         lc.compress_async(tracked, u, nbits, sbuf, ws)
@@ -389,12 +398,75 @@ def run_ours(args, rank, world, local_rank):
         "recover_k1": {"ms": rec1_ms, "alg_gbs": (8.0 * n + stream_bytes[0]) / (rec1_ms * 1e-3) / 1e9,
                        "frac_of_peak": (8.0 * n + stream_bytes[0]) / (rec1_ms * 1e-3) / 1e9 / peak},
         "ratio": {"stream": 4.0 * n / stream_bytes[-1], "bits_per_element": 8.0 * sbar[-1]},
+        "size_model": size_model,
         "roofline": roofline, "clocks": clocks, "e2e": e2e,
         "gpu_launches": (3 + decode_launches) * args.steps,  # stats, table, encode + decode launches per step
     }
     if world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = time_oracle_sample(cfg, n, u0, tracked, u, streams)
     return result
+
+
+def run_sweep(args):
+    """Sizes x distributions x nbits: compress and single-stream recover times and the ratio, as CSV on stdout.
+
+    Not the benchmark line: a reference table (roofline curve over n and the degenerate cases). Vectors of
+    2^24 elements and fewer fit the 126 MB L2, so their figures are L2-resident.
+    """
+    import torch
+
+    from paper_2009_13003_b200 import binding as lc
+    from paper_2009_13003_b200 import synth
+
+    dev = torch.device("cuda", 0)
+    lc.lib()
+    peak, _ = measured_peak()
+    print("n,dist,nbits,compress_ms,recover_ms,compress_state_gbs,recover_state_gbs,compress_alg_frac,"
+          "recover_alg_frac,ratio,bits_per_element,nsym,max_len")
+    for logn in (16, 20, 24, 28, 30):
+        n = 1 << logn
+        base = synth.normal(n, 0.02, dev, synth.SEED0 + 5)
+        ws = lc.alloc_workspace(n, dev)
+        out = torch.empty_like(base)
+        for dist in synth.SWEEP_DISTS:
+            b = torch.zeros_like(base) if dist.startswith("one_exp") else base
+            cur = b + synth.sweep_delta(dist, n, dev, synth.SEED0 + 5 + logn)
+            for nbits in ((2, 3, 4, 5, 6, 8) if logn <= 24 else (2, 5, 8)):
+                sbuf = lc.alloc_stream(n, nbits, dev)
+                times = {"c": [], "r": []}
+                for it in range(3 + 5):
+                    e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                    e[0].record()
+                    lc.compress_async(b, cur, nbits, sbuf, ws)
+                    e[1].record()
+                    torch.cuda.synchronize()
+                    if lc.last_status(ws) != 0:
+                        raise SystemExit("compress failed on %s n=%d nbits=%d: status %d" % (dist, n, nbits, lc.last_status(ws)))
+                    info = lc.stream_info(sbuf)
+                    s = sbuf[: info.total_bytes]
+                    e[1].record()
+                    lc.recover_async(b, [s], out, ws)
+                    e[2].record()
+                    torch.cuda.synchronize()
+                    if it >= 3:
+                        times["r"].append(e[1].elapsed_time(e[2]))
+                    e[0].record()
+                    lc.compress_async(b, cur, nbits, sbuf, ws)
+                    e[1].record()
+                    torch.cuda.synchronize()
+                    if it >= 3:
+                        times["c"].append(e[0].elapsed_time(e[1]))
+                assert lc.last_status(ws) == 0
+                c_ms, r_ms = statistics.median(times["c"]), statistics.median(times["r"])
+                sb = int(info.total_bytes)
+                print("%d,%s,%d,%.4f,%.4f,%.1f,%.1f,%.3f,%.3f,%.2f,%.3f,%d,%d" % (
+                    n, dist, nbits, c_ms, r_ms, 4 * n / c_ms / 1e6, 4 * n / r_ms / 1e6,
+                    (8.0 * n + sb) / c_ms / 1e6 / peak, (8.0 * n + sb) / r_ms / 1e6 / peak,
+                    4.0 * n / sb, 8.0 * sb / n, info.nsym, info.max_len), flush=True)
+                del sbuf
+            del cur
+        del base, ws, out
+        torch.cuda.empty_cache()
 
 
 def main():
@@ -407,7 +479,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default=WORKLOAD, choices=["lenet5", "resnet18", "vgg16", "xfmr1p3b"],
                     help="synthetic config; the metric is quoted on the default")
+    ap.add_argument("--sweep", action="store_true", help="print the size x distribution x nbits table (CSV) instead")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         rank = int(os.environ.get("RANK", "0"))
         res = run_reference(args, rank)

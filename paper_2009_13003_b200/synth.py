@@ -44,7 +44,8 @@ def normal(n, std, device, seed):
 def laplace(n, scale, device, seed):
     def draw(m, g):
         u = torch.rand(m, generator=g, device=device) - 0.5
-        return -scale * torch.sign(u) * torch.log1p(-2.0 * u.abs())
+        # rand() can return exactly 0, i.e. |u| = 0.5 and an infinite draw: keep |u| below one half
+        return -scale * torch.sign(u) * torch.log1p(-2.0 * u.abs().clamp_(max=0.5 - 2.0 ** -25))
 
     return _fill(n, device, seed, draw)
 
@@ -72,7 +73,8 @@ def one_exponent(n, lo_pow, device, seed, two_sign):
 
     def draw(m, g):
         mag = (1.0 + torch.rand(m, generator=g, device=device)) * (2.0 ** lo_pow)
-        mag = torch.clamp(mag, max=math.nextafter(2.0 ** (lo_pow + 1), 0.0))
+        top = torch.tensor(2.0 ** (lo_pow + 1), dtype=torch.float32)
+        mag = torch.clamp(mag, max=float(torch.nextafter(top, torch.tensor(0.0))))  # largest fp32 below 2^(lo_pow+1)
         if not two_sign:
             return mag
         sgn = torch.randint(0, 2, (m,), generator=g, device=device, dtype=torch.int8)
