@@ -1,0 +1,186 @@
+"""The pins are sharp: a plausible mistake planted in a copy of the oracle (on the CPU) makes some pin fail.
+
+Each mutation edits one line of a temporary copy of ``oracle/lc_oracle.cpp``, builds it with g++ and runs a
+compact set of pin checks against it. The real oracle must pass the same checks. Nothing here touches the
+CUDA path or a GPU.
+"""
+import ctypes as C
+import itertools
+import os
+import subprocess
+import tempfile
+
+import numpy as np
+import pytest
+
+from conftest import ROOT, load_golden
+
+SRC = os.path.join(ROOT, "oracle", "lc_oracle.cpp")
+
+MUTATIONS = [
+    ("delta sign", "const float d = cur[i] - base[i];", "const float d = base[i] - cur[i];"),
+    ("exponent mask", "const int E = static_cast<int>((u >> 23) & 255u);", "const int E = static_cast<int>((u >> 23) & 127u);"),
+    ("sign ignored in key", "return 256 * s + E;", "return E;"),
+    ("min never updated", "if (d < b.vmin) b.vmin = d;", "if (d > b.vmin) b.vmin = d;"),
+    ("selection ascending", "for (int E = 254; E >= 1; --E) {", "for (int E = 1; E <= 254; ++E) {"),
+    ("negative before positive", "for (int s = 0; s <= 1; ++s) {\n      const int key = 256 * s + E;\n      if (buckets[key].count > 0 && kept < keep_max)",
+     "for (int s = 1; s >= 0; --s) {\n      const int key = 256 * s + E;\n      if (buckets[key].count > 0 && kept < keep_max)"),
+    ("keeps 2^x buckets", "const int keep_max = (1 << nbits) - 1;", "const int keep_max = (1 << nbits);"),
+    ("mean of min and max dropped", "(static_cast<double>(vmin) + static_cast<double>(vmax)) * 0.5", "static_cast<double>(vmax)"),
+    ("midrange in float", "const double mid = (static_cast<double>(vmin) + static_cast<double>(vmax)) * 0.5;",
+     "const double mid = static_cast<double>((vmin + vmax) * 0.5f);"),
+    ("huffman tie: internal first", "nodes[front_a].weight <= nodes[front_b].weight", "nodes[front_a].weight < nodes[front_b].weight"),
+    ("huffman takes largest", "if (count[a] != count[b]) return count[a] < count[b];", "if (count[a] != count[b]) return count[a] > count[b];"),
+    ("canonical step", "if (r > 0) next = (next + 1) << (len[j] - prev_len);", "if (r > 0) next = (next << (len[j] - prev_len)) + 1;"),
+    ("zero count", "t->count[0] = n - kept_total;", "t->count[0] = n;"),
+    ("lane interleave", "return kChunkElems * c + kLanes * kGroup * j + kGroup * lane + e;", "return kChunkElems * c + kSteps * kGroup * lane + kGroup * j + e;"),
+    ("bit order in word", "const int pos = 31 - static_cast<int>(b & 31);\n  chunk[4 * word + pos / 8] |=", "const int pos = static_cast<int>(b & 31);\n  chunk[4 * word + pos / 8] |="),
+    ("lsb-first codes", "for (int b = t.len[symbol] - 1; b >= 0; --b) {\n          if ((t.code[symbol] >> b) & 1) set_chunk_bit(chunk, bit);",
+     "for (int b = 0; b < t.len[symbol]; ++b) {\n          if ((t.code[symbol] >> b) & 1) set_chunk_bit(chunk, bit);"),
+    ("chunk not padded to 16", "const uint64_t chunk_bytes = align16((chunk_bits + 7) / 8);", "const uint64_t chunk_bytes = (chunk_bits + 7) / 8;"),
+    ("recover subtracts", "x[i] = x[i] + parsed[j].table.rep[sym[i]];", "x[i] = x[i] - parsed[j].table.rep[sym[i]];"),
+    ("zero representative not added", "for (uint64_t i = 0; i < n; ++i) x[i] = x[i] + parsed[j].table.rep[sym[i]];",
+     "for (uint64_t i = 0; i < n; ++i) if (parsed[j].table.rep[sym[i]] != 0.0f) x[i] = x[i] + parsed[j].table.rep[sym[i]];"),
+    ("size model uses floor log", "while ((1ull << width) < k) width += 1;", "while ((2ull << width) <= k) width += 1;"),
+]
+
+
+def _build(text, workdir, name):
+    src = os.path.join(workdir, name + ".cpp")
+    lib = os.path.join(workdir, name + ".so")
+    with open(src, "w") as f:
+        f.write(text)
+    subprocess.check_call(["g++", "-std=c++17", "-O1", "-ffp-contract=off", "-fPIC", "-shared", "-o", lib, src])
+    return lib
+
+
+class _Oracle:
+    """Minimal binding of one oracle build (enough for the checks below)."""
+
+    def __init__(self, path):
+        L = C.CDLL(path)
+        u64, i32, vp = C.c_uint64, C.c_int, C.c_void_p
+        L.lco_huffman.argtypes = [vp, i32, vp, vp]
+        L.lco_model_bits.argtypes = [u64, u64, u64]
+        L.lco_model_bits.restype = u64
+        L.lco_stream_bound.argtypes = [u64, i32]
+        L.lco_stream_bound.restype = u64
+        L.lco_compress.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64)]
+        L.lco_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp]
+        L.lco_midrange.argtypes = [C.c_float, C.c_float]
+        L.lco_midrange.restype = C.c_float
+        self.L = L
+
+    def compress(self, base, cur, nbits):
+        cap = int(self.L.lco_stream_bound(base.size, nbits))
+        buf = np.zeros(cap + 64, np.uint8)
+        out = C.c_uint64(0)
+        rc = self.L.lco_compress(base.ctypes.data, cur.ctypes.data, base.size, nbits, buf.ctypes.data, cap, C.byref(out))
+        assert rc == 0
+        return buf[: out.value].copy()
+
+    def recover(self, base, streams):
+        k = len(streams)
+        ptrs = (C.c_void_p * k)(*[s.ctypes.data for s in streams])
+        sizes = (C.c_uint64 * k)(*[s.size for s in streams])
+        out = np.zeros(base.size, np.float32)
+        rc = self.L.lco_recover(base.ctypes.data, ptrs, sizes, k, base.size, out.ctypes.data)
+        assert rc == 0
+        return out
+
+    def huffman(self, counts):
+        c = np.asarray(counts, np.uint64)
+        ln = np.zeros(c.size, np.int32)
+        code = np.zeros(c.size, np.uint64)
+        assert self.L.lco_huffman(c.ctypes.data, c.size, ln.ctypes.data, code.ctypes.data) == 0
+        return ln, code
+
+
+def _brute_cost(counts):
+    best = None
+    for lens in itertools.product(range(1, len(counts) + 1), repeat=len(counts)):
+        if sum(2.0 ** -l for l in lens) <= 1.0 + 1e-12:
+            cost = sum(c * l for c, l in zip(counts, lens))
+            best = cost if best is None else min(best, cost)
+    return best
+
+
+def _pins_hold(o):
+    """A compact subset of the pins of test_oracle_pins.py; True if all hold."""
+    try:
+        for name in ("ten_elements_nbits2.txt", "skew16_nbits3.txt"):
+            g = load_golden(name)
+            base = np.zeros(g["cur"].size, np.float32)
+            if o.compress(base, g["cur"], g["nbits"]).tobytes() != g["stream"].tobytes():
+                return False
+            if o.recover(base, [g["stream"]]).view(np.uint32).tolist() != g["recovered"].view(np.uint32).tolist():
+                return False
+        if int(o.L.lco_model_bits(10, 5, 32)) != 190:
+            return False
+        for counts in ([1, 1, 1, 1, 1], [5, 1, 1, 2, 9], [3, 3, 2, 2, 1, 1]):
+            ln, code = o.huffman(counts)
+            if sum(c * int(l) for c, l in zip(counts, ln)) != _brute_cost(counts):
+                return False
+        ln, code = o.huffman([1, 1, 1, 1, 1])
+        if ln.tolist() != [3, 3, 2, 2, 2] or code.tolist() != [6, 7, 0, 1, 2]:
+            return False
+        # leaf against internal node of equal weight: (a+b)=2 ties with c and then with d, leaves go first,
+        # so c+d merge and every length is 2 (taking the node first gives 3,3,2,1 at the same cost)
+        if o.huffman([1, 1, 2, 2])[0].tolist() != [2, 2, 2, 2]:
+            return False
+        # exponent fields above 127 and the largest binade
+        big = np.array([8.0, 1.0, 3.0e38, 2.0 ** -125], np.float32)  # exponent fields 130, 127, 253, 2
+        s3 = o.compress(np.zeros(4, np.float32), big, 3)
+        if o.recover(np.zeros(4, np.float32), [s3]).tolist() != big.tolist():
+            return False
+        fmax = float(np.finfo(np.float32).max)
+        if float(o.L.lco_midrange(fmax, fmax)) != fmax:
+            return False
+        # adding the +0 representative turns a -0.0 base into +0.0
+        nz = np.array([0x80000000, 0x3F800000], np.uint32).view(np.float32)
+        s2 = o.compress(nz, nz, 2)
+        if o.recover(nz, [s2]).view(np.uint32).tolist() != [0, 0x3F800000]:
+            return False
+        # odd mantissa sum rounds to even; recovery is a plain fp32 add on a base that needs rounding
+        lo, hi = np.array([0x3F800001], np.uint32).view(np.float32)[0], np.array([0x3F800002], np.uint32).view(np.float32)[0]
+        if np.float32(o.L.lco_midrange(float(lo), float(hi))).view(np.uint32) != 0x3F800002:
+            return False
+        rng = np.random.default_rng(7)
+        n = 6000
+        base = rng.normal(0, 0.02, n).astype(np.float32)
+        cur = (base + rng.laplace(0, 1e-3, n).astype(np.float32)).astype(np.float32)
+        s = o.compress(base, cur, 3)
+        out = o.recover(base, [s, s])
+        d = cur - base
+        once = o.recover(base, [s])
+        dq = once - base
+        kept = np.abs(dq) > 0
+        if not np.all(np.sign(dq[kept]) == np.sign(d[kept])):
+            return False
+        if not np.array_equal(out.view(np.uint32), o.recover(once, [s]).view(np.uint32)):
+            return False
+        big = np.abs(d) >= np.abs(d).max() / 2  # the largest deltas are always kept and land within a binade
+        if not np.all(np.abs(dq[big] - d[big]) <= np.abs(d[big]) / 2 + 1e-12):
+            return False
+        return True
+    except AssertionError:
+        return False
+
+
+@pytest.fixture(scope="module")
+def workdir():
+    with tempfile.TemporaryDirectory() as d:
+        yield d
+
+
+def test_unmodified_oracle_passes_the_compact_pins(workdir):
+    assert _pins_hold(_Oracle(_build(open(SRC).read(), workdir, "clean")))
+
+
+@pytest.mark.parametrize("name,old,new", MUTATIONS, ids=[m[0] for m in MUTATIONS])
+def test_planted_mistake_is_caught(workdir, name, old, new):
+    text = open(SRC).read()
+    assert text.count(old) >= 1, "mutation target not found: " + name
+    mutated = text.replace(old, new, 1)
+    lib = _build(mutated, workdir, "mut_" + "".join(ch if ch.isalnum() else "_" for ch in name))
+    assert not _pins_hold(_Oracle(lib)), "no pin noticed: " + name
