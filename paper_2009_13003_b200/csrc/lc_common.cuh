@@ -36,7 +36,9 @@ __host__ __device__ inline StreamLayout stream_layout(uint64_t n, uint32_t nsym)
 
 // ---- statistics pass -> encode pass hand-over ("key plane") -----------------------------------
 // The statistics kernel leaves one byte per element in the workspace so that the encode pass reads
-// 1 byte per element instead of 8: (sign << 7) | (exponent field & 127). That identifies the bucket as
+// 1 byte per element instead of 8: ((exponent field & 127) << 1) | sign (the sign in bit 0, so that the two
+// signs of an exponent and 16 neighbouring exponents fall into 32 different banks of a table indexed by
+// this byte). That identifies the bucket as
 // long as every exponent field is below 128, i.e. every |delta| < 2; if some delta is larger (the
 // statistics tell), the encode pass ignores the plane and recomputes the keys from base and cur.
 // A *unit* is 1024 consecutive elements = 8 steps of one chunk, handled by one warp iteration:

@@ -18,9 +18,11 @@
 //      decoupled look-back over per-tile descriptors (per-chunk descriptors were tried: with thousands
 //      of chunks in flight every look-back walks too far back);
 //   E. the chunk image is copied to the payload with coalesced 16-byte stores.
-// Tiles are handed out by an atomic ticket, so every tile a CTA waits for in D has already been
-// started by a running CTA. The wait is bounded all the same: after kSpinLimit polls the CTA records
-// LC_ERR_TIMEOUT, marks its tile aborted (successors see that at once and abort too) and moves on.
+// The loop is software-pipelined: D and E of a tile run after A and B of the CTA's next tile (whose C follows
+// once E has freed the image area), and D is done by whichever warp finishes coding first (see the loop). Tiles are handed out by an atomic ticket, so
+// every tile a CTA waits for in D has already been started by a running CTA, and coding never waits for
+// anything. The wait is bounded all the same: after kSpinLimit polls the CTA records LC_ERR_TIMEOUT, marks
+// its tile aborted (successors see that at once and abort too) and moves on.
 //
 // Rare cases take a compact two-pass path (lengths, then bits ORed in place): the ragged last chunk,
 // codes longer than 32 bits, a lane or chunk that outgrows its shared-memory area, and vectors with an
@@ -38,6 +40,7 @@ constexpr int kEncThreads = kEncWarps * 32;
 // all 8 while an average chunk fits half of a 6 KB share (column matrix + chunk image), else 4, 2 or 1.
 constexpr uint32_t kEncSmem = 48 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr int kLookBack = 8;  // look-back sub-windows of 32 tile descriptors read per round
 
 constexpr uint32_t kPackedLenShift = 26;                      // packed entry: length << 26 | code
 constexpr uint32_t kPackedCodeMask = (1u << kPackedLenShift) - 1;
@@ -61,7 +64,7 @@ struct KeySource {
       return __float_as_uint(__fsub_rn(cur[i], base[i])) >> 23;
     }
     const uint32_t b = plane[c * kChunkElems + (j >> 2) * 512 + lane * 16 + (j & 3) * 4 + e];
-    return ((b & 128u) << 1) | (b & 127u);
+    return ((b & 1u) << 8) | (b >> 1);
   }
 };
 
@@ -155,16 +158,18 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
               uint8_t* __restrict__ stream) {
   extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ Tables tb;
-  __shared__ uint32_t s_chunk_bytes[kEncWarps];
+  __shared__ uint32_t s_chunk_bytes[2][kEncWarps];  // [half][warp]: the pending tile and the one being coded
   __shared__ uint32_t s_tile;
-  __shared__ unsigned long long s_tile_base;
+  __shared__ uint32_t s_lane_start[2][kEncThreads];  // only for chunks too large for the image area
+  __shared__ unsigned long long s_tile_base, s_tile_end;
   __shared__ int s_abort;
+  __shared__ uint32_t s_arrived[2];  // warps that have coded their chunk of the tile in this half
 
   if (ctl->status != 0) return;  // the table pass rejected the vector
 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (uint32_t b = tid; b < 256; b += kEncThreads) {
-    const EncEntry e = ctl->enc[((b & 128u) << 1) | (b & 127u)];
+    const EncEntry e = ctl->enc[((b & 1u) << 8) | (b >> 1)];
     tb.full[b] = make_uint2(e.code_lo, e.len);
     tb.packed[b] = e.len <= kPackedMaxLen ? (e.len << kPackedLenShift) | e.code_lo : kPackedLong << kPackedLenShift;
   }
@@ -222,17 +227,30 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
 
   const uint64_t ntiles = (nchunks + active - 1) / active;
 
+  // The loop is software-pipelined over tiles: a tile's offset is looked up, and its image copied out, only
+  // after the *next* tile has been coded. Every earlier tile needs its size before this one can be placed, and
+  // with hundreds of tiles in flight some predecessor is always late; looking back right after coding made the
+  // whole CTA wait for that straggler for a third of its time. One coding phase later the predecessors' sizes
+  // are there. The pending tile lives in the warps' image areas, which coding (phase A) does not touch.
+  // What the pending tile needs later is kept in shared memory (its chunk sizes, the lanes' start bits) or
+  // recomputed from its number: phase A has no registers to spare.
+  bool p_have = false;
+  uint32_t p_tile = 0, p_buf = 0;
+
+  if (tid == 0) {
+    s_tile = atomicAdd(&ctl->ticket, 1u);
+    s_abort = 0;
+    s_arrived[0] = s_arrived[1] = 0;
+  }
   while (true) {
-    __syncthreads();  // previous tile is done with s_tile, s_chunk_bytes and the shared areas
-    if (tid == 0) {
-      s_tile = atomicAdd(&ctl->ticket, 1u);
-      s_abort = 0;
-    }
-    __syncthreads();
+    __syncthreads();  // the ticket taken during the previous iteration is visible; that iteration is done
+                      // with the other half of s_chunk_bytes
     const uint64_t tile = s_tile;
-    if (tile >= ntiles) break;
+    const bool have = tile < ntiles;
+    if (!have && !p_have) break;
+    const uint32_t buf = p_buf ^ 1u;
     const uint64_t c = tile * active + warp;
-    const bool valid = warp < active && c < nchunks;
+    const bool valid = have && warp < active && c < nchunks;
     bool fast = valid && fast_chunk(c);
 
     // ---- A: code the lane's elements into its column. Lookups run one row (4 elements) ahead of the
@@ -280,18 +298,122 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     const uint32_t chunk_bits = __shfl_sync(0xffffffffu, incl, 31);
     const uint32_t chunk_bytes = valid ? (uint32_t)align_up((chunk_bits + 7) / 8, kPayloadAlign) : 0u;
     const bool staged = chunk_bytes <= image_words * 4;
-    if (lane == 0) s_chunk_bytes[warp] = chunk_bytes;
-    __syncthreads();
-    unsigned long long tile_bytes = 0;
+    if (!staged) s_lane_start[buf][tid] = lane_start;
+    // The warp that gets here first looks up the pending tile's offset (D) while the others are still coding.
+    uint32_t arrival = 0;
+    if (lane == 0) {
+      s_chunk_bytes[buf][warp] = chunk_bytes;
+      arrival = atomicAdd(&s_arrived[buf], 1u);
+    }
+    arrival = __shfl_sync(0xffffffffu, arrival, 0);
+
+    // ---- D: exclusive prefix of the pending tile by decoupled look-back
+    if (p_have && arrival == 0) {
+      unsigned long long part = 0;  // this lane's share of the sum
+      bool abort = false;
+      if (p_tile > 0) {
+        long long look = (long long)p_tile - 1;
+        uint32_t spins = 0;
+        bool done = false;
+        while (!done && !abort) {
+          // a round reads the kLookBack * 32 descriptors before `look` at once: the nearest tile that
+          // already knows its prefix is about one coding phase of tickets back
+          unsigned long long st[kLookBack];
 #pragma unroll
-    for (int w = 0; w < (int)kEncWarps; ++w) tile_bytes += s_chunk_bytes[w];
+          for (int u = 0; u < kLookBack; ++u) {
+            const long long idx = look - 32 * u - lane;
+            st[u] = (kTilePrefix << kTileFlagShift);  // tiles before the first: prefix 0
+            if (idx >= 0) st[u] = ld_tile(&tiles[idx]);
+          }
+          bool retry = false;
+#pragma unroll
+          for (int u = 0; u < kLookBack; ++u) {
+            if (done || abort || retry) continue;
+            const uint32_t flag = (uint32_t)(st[u] >> kTileFlagShift);
+            const uint32_t m_prefix = __ballot_sync(0xffffffffu, flag == kTilePrefix);
+            const uint32_t m_other = __ballot_sync(0xffffffffu, flag != kTilePrefix && flag != kTileAggregate);
+            const int first_prefix = m_prefix ? __ffs(m_prefix) - 1 : 32;
+            const uint32_t relevant = first_prefix < 32 ? (0xffffffffu >> (31 - first_prefix)) : 0xffffffffu;
+            if (m_other & relevant) {
+              // a tile without a size yet, or an aborted one
+              if (__ballot_sync(0xffffffffu, flag == kTileAbort) & relevant) abort = true;
+              else retry = true;  // poll again from `look`, which already skips the complete sub-windows
+            } else {
+              if ((int)lane <= first_prefix) part += st[u] & kTileValueMask;
+              if (first_prefix < 32) done = true;
+              else look -= 32;
+            }
+          }
+          if (retry) {
+            if (++spins > kSpinLimit) abort = true;
+            else __nanosleep(40);
+          }
+        }
+      }
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+      if (lane == 0) {
+        if (abort) {
+          set_status(&ctl->status, LC_ERR_TIMEOUT);
+          st_tile(&tiles[p_tile], kTileAbort << kTileFlagShift);
+          s_abort = 1;
+        } else {
+          unsigned long long p_tile_bytes = 0;
+#pragma unroll
+          for (int w = 0; w < (int)kEncWarps; ++w) p_tile_bytes += s_chunk_bytes[p_buf][w];
+          if (p_tile > 0) st_tile(&tiles[p_tile], (kTilePrefix << kTileFlagShift) | (part + p_tile_bytes));
+          s_abort = 0;
+          s_tile_base = part;
+          s_tile_end = part + p_tile_bytes;
+        }
+      }
+    }
+    __syncthreads();  // all chunk sizes of the new tile, and the pending tile's offset, are known
     if (tid == 0) {
-      const unsigned long long flag = tile == 0 ? kTilePrefix : kTileAggregate;
-      st_tile(&tiles[tile], (flag << kTileFlagShift) | tile_bytes);
-      if (tile == 0) s_tile_base = 0;
+      s_arrived[p_buf] = 0;  // the other half's counter, for the next iteration
+      if (have) {
+        unsigned long long tile_bytes = 0;
+#pragma unroll
+        for (int w = 0; w < (int)kEncWarps; ++w) tile_bytes += s_chunk_bytes[buf][w];
+        const unsigned long long flag = tile == 0 ? kTilePrefix : kTileAggregate;
+        st_tile(&tiles[tile], (flag << kTileFlagShift) | tile_bytes);
+      }
     }
 
-    // ---- C: assemble the chunk image in shared memory
+    // ---- E: write the pending tile's chunks and their index entries
+    if (p_have && !s_abort) {
+      unsigned long long chunk_off = s_tile_base;
+      for (uint32_t w = 0; w < warp; ++w) chunk_off += s_chunk_bytes[p_buf][w];
+      const uint64_t p_c = (uint64_t)p_tile * active + warp;
+      const uint32_t p_chunk_bytes = s_chunk_bytes[p_buf][warp];
+      const bool p_staged = p_chunk_bytes <= image_words * 4;
+      if (warp < active && p_c < nchunks) {
+        if (lane == 0) chunk_index[p_c] = chunk_off;
+        uint4* dst4 = reinterpret_cast<uint4*>(payload + chunk_off);
+        if (p_staged) {
+          const uint4* im4 = reinterpret_cast<const uint4*>(image);
+          for (uint32_t k = lane; k < p_chunk_bytes / 16; k += 32) dst4[k] = im4[k];
+        } else {
+          // chunk larger than the image area: OR the bits straight into (zeroed) global memory.
+          for (uint32_t k = lane; k < p_chunk_bytes / 16; k += 32) dst4[k] = make_uint4(0, 0, 0, 0);
+          __threadfence_block();
+          __syncwarp();
+          chunk_slow(ctl->enc, ks, p_c, lane, n, reinterpret_cast<uint32_t*>(dst4), s_lane_start[p_buf][tid]);
+        }
+      }
+      if (p_tile == ntiles - 1 && tid == 0) {
+        const unsigned long long payload_bytes = s_tile_end;
+        chunk_index[nchunks] = payload_bytes;
+        *reinterpret_cast<unsigned long long*>(stream + 48) = L.payload_off + payload_bytes;
+      }
+    }
+    if (!have) break;
+    // The next ticket is taken now, so that the round trip overlaps the rest of this iteration. (Taking it
+    // earlier would only make the tile look late to its successors: its size cannot appear before it is coded.)
+    if (tid == 0) s_tile = atomicAdd(&ctl->ticket, 1u);
+    __syncwarp();  // the warp's image area is free again
+
+    // ---- C: assemble the new tile's chunk image in shared memory
     if (valid && staged) {
       uint4* im4 = reinterpret_cast<uint4*>(image);
       for (uint32_t k = lane; k < chunk_bytes / 16; k += 32) im4[k] = make_uint4(0, 0, 0, 0);
@@ -311,78 +433,10 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
         chunk_slow(ctl->enc, ks, c, lane, n, image, lane_start);
       }
     }
-
-    // ---- D: exclusive prefix of the tile by decoupled look-back (warp 0)
-    if (warp == 0 && tile > 0) {
-      unsigned long long excl = 0;
-      long long look = (long long)tile - 1;
-      uint32_t spins = 0;
-      bool abort = false;
-      while (true) {
-        const long long idx = look - lane;
-        unsigned long long st = (kTilePrefix << kTileFlagShift);  // tiles before the first: prefix 0
-        if (idx >= 0) st = ld_tile(&tiles[idx]);
-        const uint32_t flag = (uint32_t)(st >> kTileFlagShift);
-        const uint32_t m_prefix = __ballot_sync(0xffffffffu, flag == kTilePrefix);
-        const uint32_t m_invalid = __ballot_sync(0xffffffffu, flag == kTileInvalid);
-        const uint32_t m_abort = __ballot_sync(0xffffffffu, flag == kTileAbort);
-        const int first_prefix = m_prefix ? __ffs(m_prefix) - 1 : 32;
-        const uint32_t relevant = first_prefix < 32 ? (0xffffffffu >> (31 - first_prefix)) : 0xffffffffu;
-        if (m_abort & relevant) {
-          abort = true;
-          break;
-        }
-        if (m_invalid & relevant) {
-          if (++spins > kSpinLimit) {
-            abort = true;
-            break;
-          }
-          __nanosleep(40);
-          continue;
-        }
-        unsigned long long v = ((int)lane <= first_prefix) ? (st & kTileValueMask) : 0ull;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-        excl += v;
-        if (first_prefix < 32) break;
-        look -= 32;
-      }
-      if (lane == 0) {
-        if (abort) {
-          set_status(&ctl->status, LC_ERR_TIMEOUT);
-          st_tile(&tiles[tile], kTileAbort << kTileFlagShift);
-          s_abort = 1;
-        } else {
-          st_tile(&tiles[tile], (kTilePrefix << kTileFlagShift) | (excl + tile_bytes));
-          s_tile_base = excl;
-        }
-      }
-    }
-    __syncthreads();
-    if (s_abort) continue;
-
-    // ---- E: write the chunk and its index entry
-    unsigned long long chunk_off = s_tile_base;
-    for (uint32_t w = 0; w < warp; ++w) chunk_off += s_chunk_bytes[w];
-    if (valid) {
-      if (lane == 0) chunk_index[c] = chunk_off;
-      uint4* dst4 = reinterpret_cast<uint4*>(payload + chunk_off);
-      if (staged) {
-        const uint4* im4 = reinterpret_cast<const uint4*>(image);
-        for (uint32_t k = lane; k < chunk_bytes / 16; k += 32) dst4[k] = im4[k];
-      } else {
-        // chunk larger than the image area: OR the bits straight into (zeroed) global memory.
-        for (uint32_t k = lane; k < chunk_bytes / 16; k += 32) dst4[k] = make_uint4(0, 0, 0, 0);
-        __threadfence_block();
-        __syncwarp();
-        chunk_slow(ctl->enc, ks, c, lane, n, reinterpret_cast<uint32_t*>(dst4), lane_start);
-      }
-    }
-    if (tile == ntiles - 1 && tid == 0) {
-      const unsigned long long payload_bytes = s_tile_base + tile_bytes;
-      chunk_index[nchunks] = payload_bytes;
-      *reinterpret_cast<unsigned long long*>(stream + 48) = L.payload_off + payload_bytes;
-    }
+    __syncwarp();
+    p_have = true;
+    p_tile = (uint32_t)tile;
+    p_buf = buf;
   }
 }
 

@@ -7,7 +7,8 @@
 // Bound: HBM. 8 bytes per element must be read; 1 byte per element is written.
 //
 // Design for a skewed histogram (a handful of exponents hold almost all elements):
-//  * counts live in shared memory as cnt[key][lane]: every lane of a warp owns its own column, so the
+//  * counts live in shared memory as cnt[slot][lane] (slot = the key with the sign moved to bit 0):
+//    every lane of a warp owns its own column, so the
 //    32 atomics of one warp instruction always hit 32 different banks and never the same address,
 //    whatever the keys are;
 //  * min / max are kept per key as a pair of running maxima (of ~bits and of bits: inside one key the
@@ -33,27 +34,29 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) {
   return v;
 }
 
-// Top byte = (sign << 7) | (exponent field & 127): bit 31 stays, bits 29..23 move up by one.
-__device__ __forceinline__ uint32_t plane_bits(uint32_t bits) {
-  return ((bits << 1) & 0x7F000000u) | (bits & 0x80000000u);
-}
+// Slot of a delta's bucket in the shared-memory tables: (exponent field << 1) | sign. The two signs of one
+// exponent are neighbours and 8 consecutive exponents fill the 16 bank pairs of a 64-bit access exactly once,
+// so the few hot buckets of a vector (neighbouring exponents, both signs) rarely meet in a bank. The low byte
+// of the slot is the element's byte in the key plane.
+__device__ __forceinline__ uint32_t slot_of(uint32_t bits) { return ((bits >> 22) & 0x1FEu) | (bits >> 31); }
+__device__ __forceinline__ uint32_t key_of_slot(uint32_t slot) { return ((slot & 1u) << 8) | (slot >> 1); }
 
 struct Acc {
   uint32_t* cnt_lane;  // &cnt[lane]
   uint2* mm;
-  __device__ __forceinline__ void improve(uint32_t bits, uint32_t key, uint2 cur) {
-    if (~bits > cur.x) atomicMax(&mm[key].x, ~bits);
-    if (bits > cur.y) atomicMax(&mm[key].y, bits);
+  __device__ __forceinline__ void improve(uint32_t bits, uint32_t slot, uint2 cur) {
+    if (~bits > cur.x) atomicMax(&mm[slot].x, ~bits);
+    if (bits > cur.y) atomicMax(&mm[slot].y, bits);
   }
   __device__ __forceinline__ void add(uint32_t bits) {
-    const uint32_t key = bits >> 23;
-    atomicAdd(cnt_lane + key * 32, 1u);
-    improve(bits, key, mm[key]);
+    const uint32_t slot = slot_of(bits);
+    atomicAdd(cnt_lane + slot * 32, 1u);
+    improve(bits, slot, mm[slot]);
   }
   // Four elements at once: the four reads of the running min / max pairs go out together, and one test
   // covers all eight comparisons, because after the first few elements none of them ever holds.
-  __device__ __forceinline__ void add4(uint32_t d0, uint32_t d1, uint32_t d2, uint32_t d3) {
-    const uint32_t k0 = d0 >> 23, k1 = d1 >> 23, k2 = d2 >> 23, k3 = d3 >> 23;
+  __device__ __forceinline__ void add4(uint32_t d0, uint32_t d1, uint32_t d2, uint32_t d3, uint32_t k0, uint32_t k1,
+                                       uint32_t k2, uint32_t k3) {
     const uint2 c0 = mm[k0], c1 = mm[k1], c2 = mm[k2], c3 = mm[k3];
     atomicAdd(cnt_lane + k0 * 32, 1u);
     atomicAdd(cnt_lane + k1 * 32, 1u);
@@ -102,11 +105,11 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
         const uint32_t d1 = __float_as_uint(__fsub_rn(c[r].y, b[r].y));
         const uint32_t d2 = __float_as_uint(__fsub_rn(c[r].z, b[r].z));
         const uint32_t d3 = __float_as_uint(__fsub_rn(c[r].w, b[r].w));
-        acc.add4(d0, d1, d2, d3);
-        // plane byte = sign, then the low 7 bits of the exponent field: byte 3 of plane_bits(); gather the
-        // four into one word, slot e in byte e.
-        const uint32_t lo = __byte_perm(plane_bits(d0), plane_bits(d1), 0x0073);
-        const uint32_t hi = __byte_perm(plane_bits(d2), plane_bits(d3), 0x0073);
+        const uint32_t k0 = slot_of(d0), k1 = slot_of(d1), k2 = slot_of(d2), k3 = slot_of(d3);
+        acc.add4(d0, d1, d2, d3, k0, k1, k2, k3);
+        // plane byte = low byte of the slot; gather the four into one word, element e in byte e.
+        const uint32_t lo = __byte_perm(k0, k1, 0x0040);
+        const uint32_t hi = __byte_perm(k2, k3, 0x0040);
         ew[r] = __byte_perm(lo, hi, 0x5410);
       }
     } else {
@@ -121,7 +124,7 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
             d = __float_as_uint(__fsub_rn(cur[i], base[i]));
             acc.add(d);
           }
-          word |= (plane_bits(d) >> 24) << (8 * e);
+          word |= (slot_of(d) & 255u) << (8 * e);
         }
         ew[r] = word;
       }
@@ -133,14 +136,15 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
   __syncthreads();
 
   // fold the 32 lane columns of each key and merge into the global bins.
-  for (uint32_t key = threadIdx.x; key < kKeys; key += kStatsThreads) {
+  for (uint32_t slot = threadIdx.x; slot < kKeys; slot += kStatsThreads) {
     uint32_t total = 0;
 #pragma unroll 8
-    for (uint32_t l = 0; l < 32; ++l) total += cnt[key * 32 + ((l + threadIdx.x) & 31)];
+    for (uint32_t l = 0; l < 32; ++l) total += cnt[slot * 32 + ((l + threadIdx.x) & 31)];
     if (total != 0) {
+      const uint32_t key = key_of_slot(slot);
       atomicAdd(&ctl->count[key], (unsigned long long)total);
-      atomicMax(&ctl->inv_min[key], mm[key].x);
-      atomicMax(&ctl->max_bits[key], mm[key].y);
+      atomicMax(&ctl->inv_min[key], mm[slot].x);
+      atomicMax(&ctl->max_bits[key], mm[slot].y);
     }
   }
 }
