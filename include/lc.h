@@ -86,6 +86,23 @@ int lc_compress(const float* base, const float* cur, uint64_t n, int nbits, void
                 uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs);
 
 /*
+ * Compress pass that also advances the tracked state (Algorithm 1 steps 4-7 in one call): writes the same
+ * stream as lc_compress and, in its encode pass,
+ *   tracked_out_i = fl32(base_i + q_i),   q = the quantized delta the stream holds (its representative, +0 for
+ *                                         the zero bucket, added like any other value),
+ * which is bit for bit what lc_recover(base, {stream}) would return, without a second pass over the vector.
+ * tracked_out   DEVICE, n fp32, written; 16-byte aligned. May be `base` itself (the tracked state is then updated
+ *               in place: every element is read for the last time before it is written). Must not be `cur`
+ *               (LC_ERR_ARG), nor overlap base or cur in any other way.
+ * Everything else as for lc_compress. If the device rejects the vector (LC_ERR_NONFINITE) or a wait times out,
+ * tracked_out is unspecified (with tracked_out == base: partly updated only after a time-out, untouched after
+ * LC_ERR_NONFINITE).
+ */
+int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                       uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
+                       lc_cuda_stream_t cs);
+
+/*
  * lc_compress with per-kernel timing, for profiling: same arguments and result as lc_compress, but the
  * call records CUDA events around its three kernels on `cs`, waits for them, and stores the elapsed
  * milliseconds in kernel_ms (HOST float[3]: statistics pass, table pass, encode pass).

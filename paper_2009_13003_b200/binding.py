@@ -17,7 +17,7 @@ OK, ERR_ARG, ERR_CAPACITY, ERR_NONFINITE, ERR_FORMAT, ERR_MISMATCH, ERR_TIMEOUT,
 MAX_CHAIN = 8
 
 SYMBOLS = (
-    "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_timed",
+    "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_update", "lc_compress_timed",
     "lc_recover",
     "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
     "lc_debug_bins", "lc_debug_codes", "lc_compress_noalloc",
@@ -63,6 +63,7 @@ def lib():
     L.lc_workspace_bytes.argtypes = [u64]
     L.lc_workspace_bytes.restype = u64
     L.lc_compress.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp]
+    L.lc_compress_update.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
     L.lc_compress_timed.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, C.POINTER(C.c_float)]
     L.lc_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
     L.lc_stream_info.argtypes = [vp, C.POINTER(LCInfo), vp]
@@ -119,6 +120,18 @@ def compress_async(base, cur, nbits, stream, workspace):
     _check(rc, "lc_compress")
 
 
+def compress_update_async(base, cur, nbits, stream, tracked_out, workspace):
+    """Enqueues lc_compress_update on the current stream: the stream of lc_compress plus the advanced tracked state
+    in `tracked_out` (which may be `base`); no host synchronisation."""
+    _f32_cuda(base, "base"), _f32_cuda(cur, "cur"), _f32_cuda(tracked_out, "tracked_out")
+    if base.numel() != cur.numel() or base.numel() != tracked_out.numel():
+        raise ValueError("base, cur and tracked_out differ in size")
+    rc = lib().lc_compress_update(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(),
+                                  stream.numel(), tracked_out.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                  _cs(base.device))
+    _check(rc, "lc_compress_update")
+
+
 def compress_timed(base, cur, nbits, stream, workspace):
     """lc_compress with events around its kernels; returns (stats_ms, table_ms, encode_ms)."""
     ms = (C.c_float * 3)()
@@ -149,6 +162,22 @@ def compress(base, cur, nbits, stream=None, workspace=None):
     _check(last_status(workspace), "lc_compress (device)")
     info = stream_info(stream)
     return stream[: info.total_bytes]
+
+
+def compress_update(base, cur, nbits, tracked_out=None, stream=None, workspace=None):
+    """stream <- LC(cur - base) and tracked_out <- base + quantized delta in one call (``tracked_out`` may be
+    ``base``; allocated if None). Returns (stream trimmed to its size, tracked_out)."""
+    n = base.numel()
+    if stream is None:
+        stream = alloc_stream(n, nbits, base.device)
+    if workspace is None:
+        workspace = alloc_workspace(n, base.device)
+    if tracked_out is None:
+        tracked_out = torch.empty_like(base)
+    compress_update_async(base, cur, nbits, stream, tracked_out, workspace)
+    _check(last_status(workspace), "lc_compress_update (device)")
+    info = stream_info(stream)
+    return stream[: info.total_bytes], tracked_out
 
 
 def recover_async(base, streams, out, workspace):

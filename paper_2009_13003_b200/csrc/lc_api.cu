@@ -24,6 +24,28 @@ Carved carve(void* workspace, const WorkspaceLayout& W) {
   return c;
 }
 
+// lc_compress and lc_compress_update: argument checks, then memset + three kernels on `cs`.
+int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, void* stream, uint64_t stream_capacity,
+                  float* tracked_out, void* workspace, uint64_t workspace_bytes, cudaStream_t cs) {
+  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (!stream || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
+  if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
+    return LC_ERR_ARG;
+  const WorkspaceLayout W = workspace_layout(n);
+  if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
+  const Carved c = carve(workspace, W);
+
+  // control block and tile descriptors start at zero
+  cudaError_t e = cudaMemsetAsync(workspace, 0, W.plane_off, cs);
+  if (e != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), tracked_out, cs)) !=
+      cudaSuccess)
+    return LC_ERR_CUDA;
+  return LC_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -54,22 +76,16 @@ uint64_t lc_workspace_bytes(uint64_t n) { return workspace_layout(n).total; }
 
 int lc_compress(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                 uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
-  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
-  if (!stream || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
-  if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
-    return LC_ERR_ARG;
-  const WorkspaceLayout W = workspace_layout(n);
-  if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
-  const Carved c = carve(workspace, W);
+  return compress_impl(base, cur, n, nbits, stream, stream_capacity, nullptr, workspace, workspace_bytes, cs);
+}
 
-  // control block and tile descriptors start at zero
-  cudaError_t e = cudaMemsetAsync(workspace, 0, W.plane_off, cs);
-  if (e != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), cs)) != cudaSuccess)
-    return LC_ERR_CUDA;
-  return LC_OK;
+int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                       uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
+                       lc_cuda_stream_t cs) {
+  if (n > 0 && (!tracked_out || !aligned(tracked_out, 16))) return LC_ERR_ARG;
+  if (n > 0 && tracked_out == cur) return LC_ERR_ARG;  // cur is read after parts of tracked_out are written
+  if (n == 0) tracked_out = nullptr;
+  return compress_impl(base, cur, n, nbits, stream, stream_capacity, tracked_out, workspace, workspace_bytes, cs);
 }
 
 int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
@@ -92,7 +108,7 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
   ok = ok && cudaEventRecord(ev[1], cs) == cudaSuccess;
   ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[2], cs) == cudaSuccess;
-  ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
+  ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[3], cs) == cudaSuccess;
   ok = ok && cudaEventSynchronize(ev[3]) == cudaSuccess;
   for (int i = 0; ok && i < 3; ++i) ok = cudaEventElapsedTime(&kernel_ms[i], ev[i], ev[i + 1]) == cudaSuccess;

@@ -103,8 +103,9 @@ __device__ inline void set_status(int32_t* status, int32_t code) { atomicCAS(sta
 cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
                          cudaStream_t cs);
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, cudaStream_t cs);
+// tracked_out: nullptr, or where to write base + quantized delta (may be base itself)
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
-                          const float* cur, uint64_t n, uint8_t* stream, cudaStream_t cs);
+                          const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, cudaStream_t cs);
 
 struct DecodeStreams {
   const uint8_t* ptr[4];

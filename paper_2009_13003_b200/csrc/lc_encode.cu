@@ -152,10 +152,14 @@ struct ColumnPacker {
   }
 };
 
+// UPDATE: the kernel also writes the tracked state of Algorithm 1 step 7, tracked_out = base + quantized delta
+// (fp32, the representative of the zero bucket, +0, added like any other), chunk by chunk once a chunk's coding
+// no longer needs base. tracked_out may be base itself, hence no __restrict__ on the two.
+template <bool UPDATE>
 __global__ void __launch_bounds__(kEncThreads, 4)
 encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles, const uint8_t* __restrict__ plane,
-              const float* __restrict__ base, const float* __restrict__ cur, uint64_t n,
-              uint8_t* __restrict__ stream) {
+              const float* base, const float* __restrict__ cur, uint64_t n, uint8_t* __restrict__ stream,
+              float* tracked_out) {
   extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ Tables tb;
   __shared__ uint32_t s_chunk_bytes[2][kEncWarps];  // [half][warp]: the pending tile and the one being coded
@@ -164,6 +168,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
   __shared__ unsigned long long s_tile_base, s_tile_end;
   __shared__ int s_abort;
   __shared__ uint32_t s_arrived[2];  // warps that have coded their chunk of the tile in this half
+  __shared__ uint32_t s_rep[UPDATE ? 256 : 1];  // UPDATE: representative (bit pattern) by plane byte
 
   if (ctl->status != 0) return;  // the table pass rejected the vector
 
@@ -172,6 +177,8 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     const EncEntry e = ctl->enc[((b & 1u) << 8) | (b >> 1)];
     tb.full[b] = make_uint2(e.code_lo, e.len);
     tb.packed[b] = e.len <= kPackedMaxLen ? (e.len << kPackedLenShift) | e.code_lo : kPackedLong << kPackedLenShift;
+    // the table pass has written the stream's symbol table: entry of symbol s at 64 + 16 s, representative at +4
+    if (UPDATE) s_rep[b] = *reinterpret_cast<const uint32_t*>(stream + kHeaderBytes + kTableEntryBytes * e.sym + 4);
   }
   __syncthreads();
 
@@ -407,6 +414,45 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
         *reinterpret_cast<unsigned long long*>(stream + 48) = L.payload_off + payload_bytes;
       }
     }
+    // ---- tracked state of the pending tile's chunks (everything that reads base for coding them is done)
+    if (UPDATE && p_have && !s_abort) {
+      const uint64_t p_c = (uint64_t)p_tile * active + warp;
+      if (warp < active && p_c < nchunks) {
+        if ((p_c + 1) * kChunkElems <= n && !ks.wide) {
+          const uint4* ep = reinterpret_cast<const uint4*>(plane + p_c * kChunkElems) + lane;
+          const float4* b4 = reinterpret_cast<const float4*>(base + p_c * kChunkElems) + lane;
+          float4* o4 = reinterpret_cast<float4*>(tracked_out + p_c * kChunkElems) + lane;
+#pragma unroll 2
+          for (int q = 0; q < 8; ++q) {
+            const uint4 w4 = __ldg(ep + 32 * q);  // plane bytes of steps 4q .. 4q+3
+            const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+            float4 b[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) b[r] = b4[32 * (4 * q + r)];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+              float4 x;
+              x.x = __fadd_rn(b[r].x, __uint_as_float(s_rep[__byte_perm(w[r], 0u, 0x4440)]));
+              x.y = __fadd_rn(b[r].y, __uint_as_float(s_rep[__byte_perm(w[r], 0u, 0x4441)]));
+              x.z = __fadd_rn(b[r].z, __uint_as_float(s_rep[__byte_perm(w[r], 0u, 0x4442)]));
+              x.w = __fadd_rn(b[r].w, __uint_as_float(s_rep[__byte_perm(w[r], 0u, 0x4443)]));
+              o4[32 * (4 * q + r)] = x;
+            }
+          }
+        } else {
+          // ragged last chunk, or exponents the one-byte plane does not hold: element by element
+          for (uint32_t j = 0; j < kSteps; ++j) {
+            for (uint32_t e = 0; e < kGroup; ++e) {
+              const uint64_t i = p_c * kChunkElems + 128ull * j + 4 * lane + e;
+              if (i >= n) continue;
+              const uint32_t sym = ctl->enc[ks.key(p_c, j, lane, e)].sym;
+              const uint32_t rep = *reinterpret_cast<const uint32_t*>(stream + kHeaderBytes + kTableEntryBytes * sym + 4);
+              tracked_out[i] = __fadd_rn(base[i], __uint_as_float(rep));
+            }
+          }
+        }
+      }
+    }
     if (!have) break;
     // The next ticket is taken now, so that the round trip overlaps the rest of this iteration. (Taking it
     // earlier would only make the tile look late to its successors: its size cannot appear before it is coded.)
@@ -443,25 +489,29 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
 }  // namespace
 
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
-                          const float* cur, uint64_t n, uint8_t* stream, cudaStream_t cs) {
+                          const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, cudaStream_t cs) {
   const WorkspaceLayout W = workspace_layout(n);
   if (W.nchunks == 0) return cudaSuccess;
-  static int blocks_per_sm = 0, sms = 0;
-  if (blocks_per_sm == 0) {
-    cudaError_t e = cudaFuncSetAttribute(encode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncSmem);
+  static int blocks_per_sm[2] = {0, 0}, sms = 0;
+  const int v = tracked_out ? 1 : 0;
+  if (blocks_per_sm[v] == 0) {
+    const void* fn = v ? reinterpret_cast<const void*>(encode_kernel<true>) : reinterpret_cast<const void*>(encode_kernel<false>);
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncSmem);
     if (e != cudaSuccess) return e;
     int dev = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     int bps = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, encode_kernel, kEncThreads, kEncSmem);
+    e = v ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, encode_kernel<true>, kEncThreads, kEncSmem)
+          : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, encode_kernel<false>, kEncThreads, kEncSmem);
     if (e != cudaSuccess) return e;
-    blocks_per_sm = bps > 0 ? bps : 1;
+    blocks_per_sm[v] = bps > 0 ? bps : 1;
   }
   const uint64_t want = (W.nchunks + kEncWarps - 1) / kEncWarps;
-  const uint64_t full = (uint64_t)sms * blocks_per_sm;
+  const uint64_t full = (uint64_t)sms * blocks_per_sm[v];
   const unsigned grid = (unsigned)(want < full ? want : full);
-  encode_kernel<<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream);
+  if (v) encode_kernel<true><<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, tracked_out);
+  else encode_kernel<false><<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, nullptr);
   return cudaGetLastError();
 }
 
