@@ -40,6 +40,8 @@ constexpr int kEncThreads = kEncWarps * 32;
 // all 8 while an average chunk fits half of a 6 KB share (column matrix + chunk image), else 4, 2 or 1.
 constexpr uint32_t kEncSmem = 48 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr int kUpdRows = 4;  // rows of base in flight per warp in the kernel that also writes the tracked state
+constexpr uint32_t kUpdSmem = kEncWarps * kUpdRows * 512;  // its ring, behind the kEncSmem bytes of coding areas
 constexpr int kLookBack = 8;  // look-back sub-windows of 32 tile descriptors read per round
 
 constexpr uint32_t kPackedLenShift = 26;                      // packed entry: length << 26 | code
@@ -153,10 +155,12 @@ struct ColumnPacker {
 };
 
 // UPDATE: the kernel also writes the tracked state of Algorithm 1 step 7, tracked_out = base + quantized delta
-// (fp32, the representative of the zero bucket, +0, added like any other), chunk by chunk once a chunk's coding
-// no longer needs base. tracked_out may be base itself, hence no __restrict__ on the two.
+// (fp32, the representative of the zero bucket, +0, added like any other): inside the coding loop for the chunks
+// whose coding never reads base, otherwise chunk by chunk once a chunk's coding no longer needs base.
+// tracked_out may be base itself, hence no __restrict__ on the two. Three CTAs per SM instead of four, for the
+// registers the rows of base in flight take.
 template <bool UPDATE>
-__global__ void __launch_bounds__(kEncThreads, 4)
+__global__ void __launch_bounds__(kEncThreads, UPDATE ? 3 : 4)
 encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles, const uint8_t* __restrict__ plane,
               const float* base, const float* __restrict__ cur, uint64_t n, uint8_t* __restrict__ stream,
               float* tracked_out) {
@@ -270,17 +274,55 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
       uint32_t g0[4], g1[4];
       uint4 cur4 = __ldg(ep);
       lookup4(cur4.x, g0);
+      // UPDATE: the tracked state of this chunk is written here, where its plane bytes are in registers; the
+      // memory traffic of the update then runs under the coding, which is bound by instruction issue. A chunk on
+      // this path never reads base for its coding (not even when it is coded again the slow way), so base may be
+      // overwritten at once. Row j of base is requested while row j - 1 is coded.
+      const float4* b4 = reinterpret_cast<const float4*>(base + c * kChunkElems) + lane;
+      float4* o4 = reinterpret_cast<float4*>(tracked_out + c * kChunkElems) + lane;
+      // Rows of base come through a ring of kUpdRows 512-byte slots per warp behind the coding areas, filled by
+      // cp.async four rows ahead: that many loads in flight per lane would not fit the registers, and the kernel's
+      // L1 is too small to help. A lane reads back only the 16 bytes it copied itself, so no barrier is needed.
+      const uint32_t ring = smem_addr(s_dyn) + kEncSmem + warp * (kUpdRows * 512) + lane * 16;
+      auto issue_row = [&](int j) {
+        if (j < (int)kSteps)
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring + (j % kUpdRows) * 512), "l"(b4 + 32 * j)
+                       : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");  // also when empty: the wait below counts groups
+      };
+      if (UPDATE) {
+#pragma unroll
+        for (int j = 0; j < kUpdRows; ++j) issue_row(j);
+      }
+      auto update_row = [&](uint32_t word, int j) {
+        asm volatile("cp.async.wait_group %0;" ::"n"(kUpdRows - 1) : "memory");  // row j has landed
+        float4 b;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(b.x), "=f"(b.y), "=f"(b.z), "=f"(b.w)
+                     : "r"(ring + (j % kUpdRows) * 512));
+        float4 x;
+        x.x = __fadd_rn(b.x, __uint_as_float(s_rep[__byte_perm(word, 0u, 0x4440)]));
+        x.y = __fadd_rn(b.y, __uint_as_float(s_rep[__byte_perm(word, 0u, 0x4441)]));
+        x.z = __fadd_rn(b.z, __uint_as_float(s_rep[__byte_perm(word, 0u, 0x4442)]));
+        x.w = __fadd_rn(b.w, __uint_as_float(s_rep[__byte_perm(word, 0u, 0x4443)]));
+        o4[32 * j] = x;
+        issue_row(j + kUpdRows);
+      };
 #pragma unroll 1
       for (int q = 0; q < 8; ++q) {
         const uint4 nxt = __ldg(ep + 32 * (q + 1 < 8 ? q + 1 : q));  // next 16 plane bytes, one step ahead
         lookup4(cur4.y, g1);
         put4(pk, cur4.x, g0);
+        if (UPDATE) update_row(cur4.x, 4 * q);
         lookup4(cur4.z, g0);
         put4(pk, cur4.y, g1);
+        if (UPDATE) update_row(cur4.y, 4 * q + 1);
         lookup4(cur4.w, g1);
         put4(pk, cur4.z, g0);
+        if (UPDATE) update_row(cur4.z, 4 * q + 2);
         lookup4(nxt.x, g0);  // first row of the next step (unused after the last step)
         put4(pk, cur4.w, g1);
+        if (UPDATE) update_row(cur4.w, 4 * q + 3);
         cur4 = nxt;
       }
       const bool overflow = pk.nb >= 32 || (pk.nb > 0 && pk.dst >= pk.lim);
@@ -417,7 +459,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     // ---- tracked state of the pending tile's chunks (everything that reads base for coding them is done)
     if (UPDATE && p_have && !s_abort) {
       const uint64_t p_c = (uint64_t)p_tile * active + warp;
-      if (warp < active && p_c < nchunks) {
+      if (warp < active && p_c < nchunks && !fast_chunk(p_c)) {  // the others were updated while they were coded
         if ((p_c + 1) * kChunkElems <= n && !ks.wide) {
           const uint4* ep = reinterpret_cast<const uint4*>(plane + p_c * kChunkElems) + lane;
           const float4* b4 = reinterpret_cast<const float4*>(base + p_c * kChunkElems) + lane;
@@ -496,13 +538,13 @@ cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t
   const int v = tracked_out ? 1 : 0;
   if (blocks_per_sm[v] == 0) {
     const void* fn = v ? reinterpret_cast<const void*>(encode_kernel<true>) : reinterpret_cast<const void*>(encode_kernel<false>);
-    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncSmem);
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncSmem + (v ? kUpdSmem : 0));
     if (e != cudaSuccess) return e;
     int dev = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     int bps = 0;
-    e = v ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, encode_kernel<true>, kEncThreads, kEncSmem)
+    e = v ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, encode_kernel<true>, kEncThreads, kEncSmem + kUpdSmem)
           : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, encode_kernel<false>, kEncThreads, kEncSmem);
     if (e != cudaSuccess) return e;
     blocks_per_sm[v] = bps > 0 ? bps : 1;
@@ -510,7 +552,7 @@ cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t
   const uint64_t want = (W.nchunks + kEncWarps - 1) / kEncWarps;
   const uint64_t full = (uint64_t)sms * blocks_per_sm[v];
   const unsigned grid = (unsigned)(want < full ? want : full);
-  if (v) encode_kernel<true><<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, tracked_out);
+  if (v) encode_kernel<true><<<grid, kEncThreads, kEncSmem + kUpdSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, tracked_out);
   else encode_kernel<false><<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, nullptr);
   return cudaGetLastError();
 }
