@@ -125,3 +125,25 @@ def test_nonfinite_delta_leaves_base_untouched(lc):
         lc.compress_update(base, cur, 4, tracked_out=base)
     assert e.value.code == lc.ERR_NONFINITE
     assert torch.equal(base.view(torch.int32), keep.view(torch.int32))
+
+
+def test_config_xfmr1p3b_full_size_in_place(lc, oracle):
+    """The benchmark's workload at full size (1,315,575,808 elements, nbits 5), tracked state advanced in place.
+
+    The stream must equal lc_compress's byte for byte (which test_gpu_parity checks against the oracle at this
+    size); the tracked state is compared in full with Algorithm 1 step 7 computed directly on the CPU.
+    """
+    from paper_2009_13003_b200 import synth
+
+    cfg = synth.CONFIGS["xfmr1p3b"]
+    n, nbits = cfg.n, cfg.nbits
+    u0 = synth.base_state(cfg, DEV)
+    u = u0 + synth.snapshot_delta(cfg, 1, DEV)
+    ws = lc.alloc_workspace(n, DEV)
+    ref = lc.compress(u0, u, nbits, workspace=ws).clone()
+    u0_h, u_h = to_np(u0), to_np(u)
+    s, tracked = lc.compress_update(u0, u, nbits, tracked_out=u0, workspace=ws)
+    assert tracked.data_ptr() == u0.data_ptr()
+    assert torch.equal(s, ref), "stream differs from lc_compress's"
+    want = oracle.apply_quantized(u0_h, u_h, nbits)
+    assert np.array_equal(to_np(tracked).view(np.uint32), want.view(np.uint32))
