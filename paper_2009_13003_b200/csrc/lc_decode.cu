@@ -241,7 +241,10 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
     } else {
       const uint2 r = canonical_lookup(S, idx, kL1Bits);
       if (r.y) ent = make_uint2(S.sorted_rep[r.x], r.y);
-      else ent = make_uint2(smem_addr(S.sub) + ((uint32_t)S.sub_of_prefix[idx] << (sub_bits + 3)), kLongCode);
+      // address of the prefix's sub-table, less the offset that the prefix bits add when the lookup indexes it
+      // with prefix and sub-table bits together (32-bit wrap-around arithmetic)
+      else ent = make_uint2(smem_addr(S.sub) + ((uint32_t)S.sub_of_prefix[idx] << (sub_bits + 3)) -
+                                ((idx << sub_bits) << 3), kLongCode);
     }
     S.l1[k] = ent;
   }
@@ -291,8 +294,7 @@ __device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane, uint3
       "mad.lo.u32 a, t, %5, %3;\n\t"
       "ld.shared.v2.u32 {%0,%1}, [a];\n\t"
       "setp.gt.u32 q, %1, 63;\n\t"
-      "shl.b32 t, %2, %6;\n\t"
-      "shr.u32 t, t, %7;\n\t"
+      "shr.u32 t, %2, %7;\n\t"         // prefix and sub-table index together: the entry's address allows for the prefix
       "mad.lo.u32 a, t, 8, %0;\n\t"
       "@q ld.shared.v2.u32 {%0,%1}, [a];\n\t"
       "}"
@@ -437,7 +439,7 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
   for (int s = 0; s < KS; ++s) {
     bits[s].seek(W[s], start[s]);
     l1lane[s] = smem_addr(S[s].l1) | ((lane & (kL1Rep - 1)) * 8u);
-    sub_shift[s] = 32 - S[s].sub_bits;
+    sub_shift[s] = 32 - kL1Bits - S[s].sub_bits;
   }
   const uint64_t e0 = c * kChunkElems + 4 * lane;
   float4 b = ldg_stream_v4(base + e0);
