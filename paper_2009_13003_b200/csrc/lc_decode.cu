@@ -285,6 +285,7 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 // prefix's sub-table, which is read by a predicated load (no branch for the few lanes that need it).
 // Written in PTX so that index scaling and base addition stay multiply-adds (they then run beside the
 // shifts and compares instead of competing with them for the integer pipe).
+template <int OFFSET>
 __device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane, uint32_t sub_shift) {
   uint2 ent;
   asm("{\n\t"
@@ -292,14 +293,14 @@ __device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane, uint3
       ".reg .pred q;\n\t"
       "shr.u32 t, %2, %4;\n\t"
       "mad.lo.u32 a, t, %5, %3;\n\t"
-      "ld.shared.v2.u32 {%0,%1}, [a];\n\t"
+      "ld.shared.v2.u32 {%0,%1}, [a+%8];\n\t"
       "setp.gt.u32 q, %1, 63;\n\t"
       "shr.u32 t, %2, %7;\n\t"         // prefix and sub-table index together: the entry's address allows for the prefix
       "mad.lo.u32 a, t, 8, %0;\n\t"
       "@q ld.shared.v2.u32 {%0,%1}, [a];\n\t"
       "}"
       : "=&r"(ent.x), "=&r"(ent.y)
-      : "r"(hi), "r"(l1lane), "n"(32 - kL1Bits), "n"(kL1Rep * 8), "n"(kL1Bits), "r"(sub_shift));
+      : "r"(hi), "r"(l1lane), "n"(32 - kL1Bits), "n"(kL1Rep * 8), "n"(kL1Bits), "r"(sub_shift), "n"(OFFSET));
   return ent;
 }
 
@@ -434,11 +435,12 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
                                                     const float* base, float* out, uint64_t c, uint32_t lane,
                                                     int32_t* status) {
   LaneBits<STAGED> bits[KS];
-  uint32_t l1lane[KS], sub_shift[KS];
+  // the streams' tables follow each other at 2 * kTableBytes: one base address, the rest as immediate offsets
+  const uint32_t l1lane = smem_addr(S[0].l1) | ((lane & (kL1Rep - 1)) * 8u);
+  uint32_t sub_shift[KS];
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
     bits[s].seek(W[s], start[s]);
-    l1lane[s] = smem_addr(S[s].l1) | ((lane & (kL1Rep - 1)) * 8u);
     sub_shift[s] = 32 - kL1Bits - S[s].sub_bits;
   }
   const uint64_t e0 = c * kChunkElems + 4 * lane;
@@ -457,11 +459,12 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
       }
       uint2 ent[KS];
       uint32_t longest = 0;
+      ent[0] = lookup_code<0>(bits[0].hi, l1lane, sub_shift[0]);
+      if (KS > 1) ent[1 % KS] = lookup_code<2 * kTableBytes>(bits[1 % KS].hi, l1lane, sub_shift[1 % KS]);
+      if (KS > 2) ent[2 % KS] = lookup_code<4 * kTableBytes>(bits[2 % KS].hi, l1lane, sub_shift[2 % KS]);
+      if (KS > 3) ent[3 % KS] = lookup_code<6 * kTableBytes>(bits[3 % KS].hi, l1lane, sub_shift[3 % KS]);
 #pragma unroll
-      for (int s = 0; s < KS; ++s) {
-        ent[s] = lookup_code(bits[s].hi, l1lane[s], sub_shift[s]);
-        longest |= ent[s].y;  // lengths are < 64, the marker is all ones
-      }
+      for (int s = 0; s < KS; ++s) longest |= ent[s].y;  // lengths are < 64, the marker is all ones
       if (__any_sync(0xffffffffu, longest > 63u)) {
 #pragma unroll
         for (int s = 0; s < KS; ++s) {
