@@ -465,7 +465,7 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
       if (KS > 3) ent[3 % KS] = lookup_code<6 * kTableBytes>(bits[3 % KS].hi, l1lane, sub_shift[3 % KS]);
 #pragma unroll
       for (int s = 0; s < KS; ++s) longest |= ent[s].y;  // lengths are < 64, the marker is all ones
-      if (__any_sync(0xffffffffu, longest > 63u)) {
+      if (__builtin_expect(__any_sync(0xffffffffu, longest > 63u), 0)) {
 #pragma unroll
         for (int s = 0; s < KS; ++s) {
           if (ent[s].y > 63u) ent[s] = make_uint2(long_code<STAGED>(bits[s], S[s], W[s], status), 0u);  // consumed
