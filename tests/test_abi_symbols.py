@@ -41,4 +41,13 @@ def test_host_argument_checks_need_no_device():
     L = binding.lib()
     assert L.lc_compress(None, None, 16, 4, None, 0, None, 0, None) == binding.ERR_ARG
     assert L.lc_recover(None, None, None, 0, 16, None, None, 0, None) == binding.ERR_ARG
+    # lc_compress_update: the tracked state must be given, aligned, and must not be cur (made-up addresses:
+    # the checks come before anything is touched)
+    base, cur, stream, ws = 0x10000, 0x20000, 0x30000, 0x40000
+    upd = lambda out, nbits=4: L.lc_compress_update(base, cur, 16, nbits, stream, 1 << 20, out, ws, 1 << 20, None)
+    assert upd(None) == binding.ERR_ARG
+    assert upd(cur) == binding.ERR_ARG
+    assert upd(0x50004) == binding.ERR_ARG
+    assert upd(0x50000, nbits=9) == binding.ERR_ARG
+    assert L.lc_compress_update(base, cur, 16, 4, stream, 8, 0x50000, ws, 1 << 20, None) == binding.ERR_CAPACITY
     assert L.lc_strerror(binding.ERR_FORMAT) == b"malformed stream"
