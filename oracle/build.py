@@ -7,7 +7,7 @@ SRC = os.path.join(HERE, "lc_oracle.cpp")
 LIB = os.path.join(HERE, "liblc_oracle.so")
 
 # -ffp-contract=off: the fp32 subtract and add of Algorithm 1 must stay plain IEEE operations.
-FLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared", "-Wall", "-Wextra"]
+FLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared", "-pthread", "-Wall", "-Wextra"]
 
 
 def build(force: bool = False) -> str:

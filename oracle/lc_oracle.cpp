@@ -13,7 +13,11 @@
 // streams written by hand from the format text, brute-force optimal prefix codes on tiny alphabets,
 // Kraft equality, entropy bound, textbook code-length cases, the integer midrange identity, the
 // paper's worked size example (Section 3.1.1: n=10, k=5 -> 190 bits, rate 1.68), round trips and the
-// chain identity of Algorithm 1.
+// chain identity of Algorithm 1. The helpers are pinned to the main functions: lco_apply_quantized to
+// lco_recover of lco_compress, lco_compress_chunks to slices of lco_compress's stream, the threaded
+// timing mode to the single-threaded bytes, lco_merge to the idempotence of quantization over a zero
+// base (the merged stream of one stream is that stream) and to Algorithm 1 step 7 applied to the
+// recovered state.
 // Parity unpinned: the whole-pipeline result on the paper's own training deltas (its figures carry
 // the only values and they are not available); only the loose size ranges of Section 4.3 apply.
 
@@ -21,6 +25,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <thread>
 #include <vector>
 
 namespace {
@@ -382,70 +387,124 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   return LCO_OK;
 }
 
-// Decodes every symbol of a stream by walking the code tree bit by bit.
-int decode_symbols(const uint8_t* s, uint64_t bytes, const Parsed& p, uint8_t* sym /*[n]*/) {
-  (void)bytes;
-  const Table& t = p.table;
-  const Layout& L = p.layout;
-  if (t.max_len == 0) {
-    int only = 0;
-    for (int j = 0; j < t.nsym; ++j)
-      if (t.count[j] > 0) only = j;
-    for (uint64_t i = 0; i < p.n; ++i) sym[i] = static_cast<uint8_t>(only);
-    return LCO_OK;
-  }
-  // Explicit binary code tree. child[bit][node] is 0 when absent, a node index when positive and
-  // -(symbol+1) at a leaf; node 0 is the root.
+// Explicit binary code tree. child[bit][node] is 0 when absent, a node index when positive and
+// -(symbol+1) at a leaf; node 0 is the root.
+struct CodeTree {
   std::vector<int> child[2] = {std::vector<int>(1, 0), std::vector<int>(1, 0)};
+  int only = 0;  // the symbol every element has when no code has a length (fewer than two used symbols)
+};
+
+int build_tree(const Table& t, CodeTree* tree) {
+  for (int j = 0; j < t.nsym; ++j)
+    if (t.count[j] > 0) tree->only = j;
   for (int j = 0; j < t.nsym; ++j) {
     if (t.len[j] == 0) continue;
     int node = 0;
     for (int b = t.len[j] - 1; b >= 0; --b) {
       const int bit = static_cast<int>((t.code[j] >> b) & 1);
       if (b == 0) {
-        child[bit][node] = -(j + 1);
+        tree->child[bit][node] = -(j + 1);
         break;
       }
-      if (child[bit][node] == 0) {
-        child[0].push_back(0);
-        child[1].push_back(0);
-        child[bit][node] = static_cast<int>(child[0].size()) - 1;
+      if (tree->child[bit][node] == 0) {
+        tree->child[0].push_back(0);
+        tree->child[1].push_back(0);
+        tree->child[bit][node] = static_cast<int>(tree->child[0].size()) - 1;
       }
-      node = child[bit][node];
+      node = tree->child[bit][node];
       if (node < 0) return LCO_ERR_FORMAT;
     }
   }
+  return LCO_OK;
+}
+
+// Decodes the symbols of chunk c by walking the code tree one bit at a time.
+int decode_chunk(const uint8_t* s, const Parsed& p, const CodeTree& tree, uint64_t c, uint8_t* sym /*[n]*/) {
+  const Layout& L = p.layout;
   const uint8_t* chunk_index = s + L.chunk_index_off;
   const uint8_t* lane_index = s + L.lane_index_off;
-  for (uint64_t c = 0; c < L.nchunks; ++c) {
-    const uint64_t off = get_le(chunk_index + 8 * c, 8);
-    const uint64_t size = get_le(chunk_index + 8 * (c + 1), 8) - off;
-    const uint8_t* chunk = s + L.payload_off + off;
-    uint64_t bit = 0;
-    for (uint64_t lane = 0; lane < kLanes; ++lane) {
-      const uint64_t lane_bits = get_le(lane_index + 2 * (kLanes * c + lane), 2);
-      const uint64_t lane_end = bit + lane_bits;
-      if (lane_end > 8 * size) return LCO_ERR_FORMAT;
-      for (uint64_t j = 0; j < kSteps; ++j) {
-        for (uint64_t e = 0; e < kGroup; ++e) {
-          const uint64_t i = element_index(c, lane, j, e);
-          if (i >= p.n) continue;
-          int node = 0;
-          while (true) {
-            if (bit >= lane_end) return LCO_ERR_FORMAT;
-            const int b = get_chunk_bit(chunk, bit);
-            bit += 1;
-            node = child[b][node];
-            if (node < 0) break;
-            if (node == 0) return LCO_ERR_FORMAT;
-          }
-          sym[i] = static_cast<uint8_t>(-node - 1);
+  const uint64_t off = get_le(chunk_index + 8 * c, 8);
+  const uint64_t size = get_le(chunk_index + 8 * (c + 1), 8) - off;
+  const uint8_t* chunk = s + L.payload_off + off;
+  uint64_t bit = 0;
+  for (uint64_t lane = 0; lane < kLanes; ++lane) {
+    const uint64_t lane_bits = get_le(lane_index + 2 * (kLanes * c + lane), 2);
+    const uint64_t lane_end = bit + lane_bits;
+    if (lane_end > 8 * size) return LCO_ERR_FORMAT;
+    for (uint64_t j = 0; j < kSteps; ++j) {
+      for (uint64_t e = 0; e < kGroup; ++e) {
+        const uint64_t i = element_index(c, lane, j, e);
+        if (i >= p.n) continue;
+        int node = 0;
+        while (true) {
+          if (bit >= lane_end) return LCO_ERR_FORMAT;
+          const int b = get_chunk_bit(chunk, bit);
+          bit += 1;
+          node = tree.child[b][node];
+          if (node < 0) break;
+          if (node == 0) return LCO_ERR_FORMAT;
         }
+        sym[i] = static_cast<uint8_t>(-node - 1);
       }
-      if (bit != lane_end) return LCO_ERR_FORMAT;
     }
+    if (bit != lane_end) return LCO_ERR_FORMAT;
   }
   return LCO_OK;
+}
+
+// Decodes every symbol of a stream, chunk after chunk.
+int decode_symbols(const uint8_t* s, uint64_t bytes, const Parsed& p, uint8_t* sym /*[n]*/) {
+  (void)bytes;
+  CodeTree tree;
+  const int rc = build_tree(p.table, &tree);
+  if (rc != LCO_OK) return rc;
+  if (p.table.max_len == 0) {
+    for (uint64_t i = 0; i < p.n; ++i) sym[i] = static_cast<uint8_t>(tree.only);
+    return LCO_OK;
+  }
+  for (uint64_t c = 0; c < p.layout.nchunks; ++c) {
+    const int rc2 = decode_chunk(s, p, tree, c, sym);
+    if (rc2 != LCO_OK) return rc2;
+  }
+  return LCO_OK;
+}
+
+// Writes header and symbol table of a stream (format sections 3.1 and 3.2).
+void write_header_and_table(uint8_t* stream, const Table& t, uint64_t n, int nbits, const Layout& L,
+                            uint64_t payload_bits, uint64_t payload_bytes) {
+  for (int j = 0; j < t.nsym; ++j) {
+    uint8_t* e = stream + L.table_off + 16 * j;
+    put_le(e, static_cast<uint64_t>(t.key[j]), 2);
+    e[2] = static_cast<uint8_t>(t.len[j]);
+    e[3] = 0;
+    put_le(e + 4, float_bits(t.rep[j]), 4);
+    put_le(e + 8, t.count[j], 8);
+  }
+  uint8_t* h = stream;
+  h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
+  put_le(h + 4, 1, 2);
+  h[6] = static_cast<uint8_t>(nbits);
+  h[7] = 0;
+  put_le(h + 8, n, 8);
+  put_le(h + 16, static_cast<uint64_t>(t.nsym), 4);
+  put_le(h + 20, static_cast<uint64_t>(t.max_len), 4);
+  put_le(h + 24, kChunkElems, 4);
+  put_le(h + 28, kLanes, 2);
+  put_le(h + 30, kGroup, 2);
+  put_le(h + 32, L.nchunks, 4);
+  put_le(h + 36, 16, 4);
+  put_le(h + 40, payload_bits, 8);
+  put_le(h + 48, L.payload_off + payload_bytes, 8);
+  put_le(h + 56, L.payload_off, 8);
+}
+
+// Runs fn(t) for t in [0, nthreads) on that many threads (the timing mode that uses all host cores).
+template <class F>
+void run_threads(int nthreads, F fn) {
+  std::vector<std::thread> pool;
+  for (int t = 1; t < nthreads; ++t) pool.emplace_back(fn, t);
+  fn(0);
+  for (auto& th : pool) th.join();
 }
 
 }  // namespace
@@ -556,32 +615,7 @@ int lco_compress(const float* base, const float* cur, uint64_t n, int nbits, uin
   }
   put_le(chunk_index + 8 * L.nchunks, payload_bytes, 8);
 
-  // table
-  for (int j = 0; j < t.nsym; ++j) {
-    uint8_t* e = stream + L.table_off + 16 * j;
-    put_le(e, static_cast<uint64_t>(t.key[j]), 2);
-    e[2] = static_cast<uint8_t>(t.len[j]);
-    e[3] = 0;
-    put_le(e + 4, float_bits(t.rep[j]), 4);
-    put_le(e + 8, t.count[j], 8);
-  }
-  // header
-  uint8_t* h = stream;
-  h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
-  put_le(h + 4, 1, 2);
-  h[6] = static_cast<uint8_t>(nbits);
-  h[7] = 0;
-  put_le(h + 8, n, 8);
-  put_le(h + 16, static_cast<uint64_t>(t.nsym), 4);
-  put_le(h + 20, static_cast<uint64_t>(t.max_len), 4);
-  put_le(h + 24, kChunkElems, 4);
-  put_le(h + 28, kLanes, 2);
-  put_le(h + 30, kGroup, 2);
-  put_le(h + 32, L.nchunks, 4);
-  put_le(h + 36, 16, 4);
-  put_le(h + 40, payload_bits, 8);
-  put_le(h + 48, L.payload_off + payload_bytes, 8);
-  put_le(h + 56, L.payload_off, 8);
+  write_header_and_table(stream, t, n, nbits, L, payload_bits, payload_bytes);
   *out_bytes = L.payload_off + payload_bytes;
   return LCO_OK;
 }
@@ -651,6 +685,124 @@ int lco_compress_chunks(const float* base, const float* cur, uint64_t n, int nbi
     for (int lane = 0; lane < 32; ++lane) lane_bits[32 * k + lane] = static_cast<uint16_t>(get_le(li + 2 * lane, 2));
     std::memcpy(payload + k * stride, chunk.data(), sz);
     bytes[k] = sz;
+  }
+  return LCO_OK;
+}
+
+
+// Checkpoint merging (Section 3.2, "Checkpoint Merging"): k consecutive checkpoints become one
+// super-step checkpoint. The paper does not say how the merged checkpoint is coded; the reading taken
+// here is the scheme applied once more to the summed change: the state the k streams recover is
+// compressed against the same base,
+//   merged = compress(base, recover(base, streams)).
+// The merged stream therefore quantizes a second time: recovering it gives a state within the
+// quantization error of, not bit-identical to, what the k streams recover.
+int lco_merge(const float* base, const uint8_t* const* streams, const uint64_t* stream_bytes, int k, uint64_t n,
+              int nbits, uint8_t* stream, uint64_t capacity, uint64_t* out_bytes) {
+  std::vector<float> recovered(n);
+  const int rc = lco_recover(base, streams, stream_bytes, k, n, recovered.data());
+  if (rc != LCO_OK) return rc;
+  return lco_compress(base, recovered.data(), n, nbits, stream, capacity, out_bytes);
+}
+
+// ---- the same two passes on several host threads (timing mode: "all host cores") -----------------
+// The steps are those of lco_compress / lco_recover; only the loops over elements and chunks are split
+// into contiguous ranges, one per thread. Bucket statistics merge by sum / min / max; chunks are coded
+// and decoded independently once the table is known. The results are byte-identical to the
+// single-threaded functions (a test checks that).
+
+int lco_compress_mt(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* stream,
+                    uint64_t capacity, uint64_t* out_bytes, int nthreads) {
+  if (nbits < 1 || nbits > 8 || n >= (1ull << 32) || nthreads < 1) return LCO_ERR_ARG;
+  if (capacity < stream_bound(n, nbits)) return LCO_ERR_CAPACITY;
+  const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
+  auto range = [&](int t, uint64_t total) {
+    return std::pair<uint64_t, uint64_t>(total * t / nthreads, total * (t + 1) / nthreads);
+  };
+  // statistics: one set of buckets per thread over a range of whole chunks, then merged
+  std::vector<std::vector<Bucket>> part(nthreads, std::vector<Bucket>(512));
+  run_threads(nthreads, [&](int t) {
+    const auto r = range(t, nchunks);
+    const uint64_t lo = std::min(n, r.first * kChunkElems), hi = std::min(n, r.second * kChunkElems);
+    delta_buckets(base + lo, cur + lo, hi - lo, part[t].data());
+  });
+  std::vector<Bucket> buckets(512);
+  for (int t = 0; t < nthreads; ++t)
+    for (int key = 0; key < 512; ++key) {
+      const Bucket& b = part[t][key];
+      Bucket& m = buckets[key];
+      if (b.count == 0) continue;
+      if (m.count == 0) {
+        m = b;
+      } else {
+        m.count += b.count;
+        if (b.vmin < m.vmin) m.vmin = b.vmin;
+        if (b.vmax > m.vmax) m.vmax = b.vmax;
+      }
+    }
+  Table t;
+  Selection sel;
+  const int rc = build_table(buckets.data(), n, nbits, &t, &sel);
+  if (rc != LCO_OK) return rc;
+  const Layout L = layout_for(n, t.nsym);
+  std::memset(stream, 0, L.payload_off);
+  // every chunk coded into a buffer of its own, then laid out in order
+  std::vector<std::vector<uint8_t>> coded(nchunks);
+  std::vector<uint64_t> bits(nchunks, 0);
+  uint8_t* lane_index = stream + L.lane_index_off;
+  run_threads(nthreads, [&](int th) {
+    const auto r = range(th, nchunks);
+    std::vector<uint8_t> chunk(kChunkElems * 8 + 16);
+    for (uint64_t c = r.first; c < r.second; ++c) {
+      const uint64_t sz = encode_chunk(base, cur, n, t, sel, c, lane_index + 2 * kLanes * c, chunk.data(), &bits[c]);
+      coded[c].assign(chunk.begin(), chunk.begin() + sz);
+    }
+  });
+  uint8_t* chunk_index = stream + L.chunk_index_off;
+  uint64_t payload_bytes = 0, payload_bits = 0;
+  for (uint64_t c = 0; c < nchunks; ++c) {
+    put_le(chunk_index + 8 * c, payload_bytes, 8);
+    std::memcpy(stream + L.payload_off + payload_bytes, coded[c].data(), coded[c].size());
+    payload_bytes += coded[c].size();
+    payload_bits += bits[c];
+  }
+  put_le(chunk_index + 8 * nchunks, payload_bytes, 8);
+  write_header_and_table(stream, t, n, nbits, L, payload_bits, payload_bytes);
+  *out_bytes = L.payload_off + payload_bytes;
+  return LCO_OK;
+}
+
+int lco_recover_mt(const float* base, const uint8_t* const* streams, const uint64_t* stream_bytes, int k,
+                   uint64_t n, float* out, int nthreads) {
+  if (k < 1 || nthreads < 1) return LCO_ERR_ARG;
+  std::vector<Parsed> parsed(static_cast<size_t>(k));
+  std::vector<CodeTree> trees(static_cast<size_t>(k));
+  for (int j = 0; j < k; ++j) {
+    int rc = parse_stream(streams[j], stream_bytes[j], &parsed[j]);
+    if (rc != LCO_OK) return rc;
+    if (parsed[j].n != n) return LCO_ERR_MISMATCH;
+    if ((rc = build_tree(parsed[j].table, &trees[j])) != LCO_OK) return rc;
+  }
+  const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
+  std::vector<uint8_t> sym(n);
+  std::vector<int> status(nthreads, LCO_OK);
+  for (uint64_t i = 0; i < n; ++i) out[i] = base[i];
+  for (int j = 0; j < k; ++j) {
+    run_threads(nthreads, [&](int th) {
+      const uint64_t c0 = nchunks * th / nthreads, c1 = nchunks * (th + 1) / nthreads;
+      for (uint64_t c = c0; c < c1; ++c) {
+        const uint64_t lo = c * kChunkElems, hi = std::min(n, lo + kChunkElems);
+        if (parsed[j].table.max_len == 0) {
+          for (uint64_t i = lo; i < hi; ++i) sym[i] = static_cast<uint8_t>(trees[j].only);
+        } else {
+          const int rc = decode_chunk(streams[j], parsed[j], trees[j], c, sym.data());
+          if (rc != LCO_OK) status[th] = rc;
+        }
+        for (uint64_t i = lo; i < hi; ++i) out[i] = out[i] + parsed[j].table.rep[sym[i]];
+      }
+    });
+    for (int th = 0; th < nthreads; ++th)
+      if (status[th] != LCO_OK) return status[th];
   }
   return LCO_OK;
 }

@@ -35,6 +35,9 @@ def lib():
         L.lco_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp]
         L.lco_apply_quantized.argtypes = [vp, vp, u64, i32, vp]
         L.lco_compress_chunks.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
+        L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
+        L.lco_compress_mt.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), i32]
+        L.lco_recover_mt.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, i32]
         _lib = L
     return _lib
 
@@ -109,8 +112,9 @@ def stream_bound(n, nbits):
     return int(lib().lco_stream_bound(n, nbits))
 
 
-def compress(base, cur, nbits):
-    """Returns the stream as a uint8 numpy array."""
+def compress(base, cur, nbits, threads=None):
+    """Returns the stream as a uint8 numpy array. ``threads``: None for the plain single-threaded pass, else the
+    number of host threads of the chunk-parallel timing mode (same bytes)."""
     base, pb = _f32(base)
     cur, pc = _f32(cur)
     if not 1 <= nbits <= 8:
@@ -118,7 +122,10 @@ def compress(base, cur, nbits):
     cap = stream_bound(base.size, nbits)
     buf = np.zeros(cap, np.uint8)
     out = C.c_uint64(0)
-    rc = lib().lco_compress(pb, pc, base.size, nbits, buf.ctypes.data, cap, C.byref(out))
+    if threads is None:
+        rc = lib().lco_compress(pb, pc, base.size, nbits, buf.ctypes.data, cap, C.byref(out))
+    else:
+        rc = lib().lco_compress_mt(pb, pc, base.size, nbits, buf.ctypes.data, cap, C.byref(out), int(threads))
     if rc < 0:
         raise OracleError(rc)
     return buf[: out.value].copy()
@@ -133,17 +140,38 @@ def decode_symbols(stream, n):
     return sym
 
 
-def recover(base, streams):
+def recover(base, streams, threads=None):
     base, pb = _f32(base)
     streams = [np.ascontiguousarray(s, dtype=np.uint8) for s in streams]
     k = len(streams)
     ptrs = (C.c_void_p * k)(*[s.ctypes.data for s in streams])
     sizes = (C.c_uint64 * k)(*[s.size for s in streams])
     out = np.zeros(base.size, np.float32)
-    rc = lib().lco_recover(pb, ptrs, sizes, k, base.size, out.ctypes.data)
+    if threads is None:
+        rc = lib().lco_recover(pb, ptrs, sizes, k, base.size, out.ctypes.data)
+    else:
+        rc = lib().lco_recover_mt(pb, ptrs, sizes, k, base.size, out.ctypes.data, int(threads))
     if rc < 0:
         raise OracleError(rc)
     return out
+
+
+def merge(base, streams, nbits):
+    """The super-step stream of Section 3.2 (checkpoint merging): compress(base, recover(base, streams))."""
+    base, pb = _f32(base)
+    streams = [np.ascontiguousarray(s, dtype=np.uint8) for s in streams]
+    k = len(streams)
+    ptrs = (C.c_void_p * k)(*[s.ctypes.data for s in streams])
+    sizes = (C.c_uint64 * k)(*[s.size for s in streams])
+    if not 1 <= nbits <= 8:
+        raise OracleError(ERR_ARG)
+    cap = stream_bound(base.size, nbits)
+    buf = np.zeros(cap, np.uint8)
+    out = C.c_uint64(0)
+    rc = lib().lco_merge(pb, ptrs, sizes, k, base.size, nbits, buf.ctypes.data, cap, C.byref(out))
+    if rc < 0:
+        raise OracleError(rc)
+    return buf[: out.value].copy()
 
 
 def apply_quantized(base, cur, nbits):

@@ -41,6 +41,21 @@ MUTATIONS = [
     ("recover subtracts", "x[i] = x[i] + parsed[j].table.rep[sym[i]];", "x[i] = x[i] - parsed[j].table.rep[sym[i]];"),
     ("zero representative not added", "for (uint64_t i = 0; i < n; ++i) x[i] = x[i] + parsed[j].table.rep[sym[i]];",
      "for (uint64_t i = 0; i < n; ++i) if (parsed[j].table.rep[sym[i]] != 0.0f) x[i] = x[i] + parsed[j].table.rep[sym[i]];"),
+    ("step 7 helper subtracts", "out[i] = base[i] + t.rep[sel.symbol_of_key[bucket_key(cur[i] - base[i])]];",
+     "out[i] = base[i] - t.rep[sel.symbol_of_key[bucket_key(cur[i] - base[i])]];"),
+    ("step 7 helper: operands of the delta swapped", "out[i] = base[i] + t.rep[sel.symbol_of_key[bucket_key(cur[i] - base[i])]];",
+     "out[i] = base[i] + t.rep[sel.symbol_of_key[bucket_key(base[i] - cur[i])]];"),
+    ("chunk helper codes another chunk", "encode_chunk(base, cur, n, t, sel, chunk_ids[k], li, chunk.data(), &bits);",
+     "encode_chunk(base, cur, n, t, sel, k, li, chunk.data(), &bits);"),
+    ("chunk helper: lane order", "lane_bits[32 * k + lane] = static_cast<uint16_t>(get_le(li + 2 * lane, 2));",
+     "lane_bits[32 * k + lane] = static_cast<uint16_t>(get_le(li + 2 * (31 - lane), 2));"),
+    ("merge: operands swapped", "return lco_compress(base, recovered.data(), n, nbits, stream, capacity, out_bytes);",
+     "return lco_compress(recovered.data(), base, n, nbits, stream, capacity, out_bytes);"),
+    ("merge: recovers from zero instead of base", "const int rc = lco_recover(base, streams, stream_bytes, k, n, recovered.data());\n  if (rc != LCO_OK) return rc;\n  return lco_compress",
+     "std::vector<float> zero(n, 0.0f);\n  const int rc = lco_recover(zero.data(), streams, stream_bytes, k, n, recovered.data());\n  if (rc != LCO_OK) return rc;\n  return lco_compress"),
+    ("threaded statistics: minimum not merged", "if (b.vmin < m.vmin) m.vmin = b.vmin;", "if (b.vmin > m.vmin) m.vmin = b.vmin;"),
+    ("threaded recovery: chunk range off by one", "const uint64_t lo = c * kChunkElems, hi = std::min(n, lo + kChunkElems);\n        if (parsed[j].table.max_len == 0)",
+     "const uint64_t lo = c * kChunkElems, hi = std::min(n, lo + kChunkElems - 1);\n        if (parsed[j].table.max_len == 0)"),
     ("size model uses floor log", "while ((1ull << width) < k) width += 1;", "while ((2ull << width) <= k) width += 1;"),
 ]
 
@@ -69,7 +84,53 @@ class _Oracle:
         L.lco_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp]
         L.lco_midrange.argtypes = [C.c_float, C.c_float]
         L.lco_midrange.restype = C.c_float
+        L.lco_apply_quantized.argtypes = [vp, vp, u64, i32, vp]
+        L.lco_compress_chunks.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
+        L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
+        L.lco_compress_mt.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), i32]
+        L.lco_recover_mt.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, i32]
         self.L = L
+
+    def apply_quantized(self, base, cur, nbits):
+        out = np.zeros(base.size, np.float32)
+        assert self.L.lco_apply_quantized(base.ctypes.data, cur.ctypes.data, base.size, nbits, out.ctypes.data) == 0
+        return out
+
+    def compress_chunks(self, base, cur, nbits, ids):
+        ids = np.asarray(ids, np.uint64)
+        stride = 4096 * 8 + 16
+        lane_bits = np.zeros((ids.size, 32), np.uint16)
+        payload = np.zeros(ids.size * stride, np.uint8)
+        sizes = np.zeros(ids.size, np.uint64)
+        assert self.L.lco_compress_chunks(base.ctypes.data, cur.ctypes.data, base.size, nbits, ids.ctypes.data, ids.size,
+                                          lane_bits.ctypes.data, payload.ctypes.data, stride, sizes.ctypes.data) == 0
+        return lane_bits, [payload[k * stride: k * stride + int(sizes[k])] for k in range(ids.size)]
+
+    def merge(self, base, streams, nbits):
+        k = len(streams)
+        ptrs = (C.c_void_p * k)(*[s.ctypes.data for s in streams])
+        sizes = (C.c_uint64 * k)(*[s.size for s in streams])
+        cap = int(self.L.lco_stream_bound(base.size, nbits))
+        buf = np.zeros(cap + 64, np.uint8)
+        out = C.c_uint64(0)
+        assert self.L.lco_merge(base.ctypes.data, ptrs, sizes, k, base.size, nbits, buf.ctypes.data, cap, C.byref(out)) == 0
+        return buf[: out.value].copy()
+
+    def compress_mt(self, base, cur, nbits, threads):
+        cap = int(self.L.lco_stream_bound(base.size, nbits))
+        buf = np.zeros(cap + 64, np.uint8)
+        out = C.c_uint64(0)
+        assert self.L.lco_compress_mt(base.ctypes.data, cur.ctypes.data, base.size, nbits, buf.ctypes.data, cap,
+                                      C.byref(out), threads) == 0
+        return buf[: out.value].copy()
+
+    def recover_mt(self, base, streams, threads):
+        k = len(streams)
+        ptrs = (C.c_void_p * k)(*[s.ctypes.data for s in streams])
+        sizes = (C.c_uint64 * k)(*[s.size for s in streams])
+        out = np.zeros(base.size, np.float32)
+        assert self.L.lco_recover_mt(base.ctypes.data, ptrs, sizes, k, base.size, out.ctypes.data, threads) == 0
+        return out
 
     def compress(self, base, cur, nbits):
         cap = int(self.L.lco_stream_bound(base.size, nbits))
@@ -161,6 +222,34 @@ def _pins_hold(o):
             return False
         big = np.abs(d) >= np.abs(d).max() / 2  # the largest deltas are always kept and land within a binade
         if not np.all(np.abs(dq[big] - d[big]) <= np.abs(d[big]) / 2 + 1e-12):
+            return False
+        # the helpers of the full-size parity tests: step 7 computed directly, single chunks of a stream
+        if not np.array_equal(o.apply_quantized(base, cur, 3).view(np.uint32), once.view(np.uint32)):
+            return False
+        nsym = int(np.frombuffer(s[16:20].tobytes(), "<u4")[0])
+        nchunks = (n + 4095) // 4096
+        ci = 64 + 16 * nsym
+        li = ci + 8 * (nchunks + 1)
+        po = int(np.frombuffer(s[56:64].tobytes(), "<u8")[0])
+        off = np.frombuffer(s[ci:li].tobytes(), "<u8")
+        lanes = np.frombuffer(s[li:li + 64 * nchunks].tobytes(), "<u2").reshape(nchunks, 32)
+        olane, opay = o.compress_chunks(base, cur, 3, [1, 0])
+        for k, c in enumerate((1, 0)):
+            if not np.array_equal(olane[k], lanes[c]) or opay[k].tobytes() != s[po + int(off[c]): po + int(off[c + 1])].tobytes():
+                return False
+        # checkpoint merging: over a zero base a single stream merges into itself; in general the merged stream
+        # recovers the once-more-quantized change on top of the base
+        z = np.zeros(n, np.float32)
+        sz = o.compress(z, cur, 3)
+        if o.merge(z, [sz], 3).tobytes() != sz.tobytes():
+            return False
+        m = o.merge(base, [s, s], 3)
+        if not np.array_equal(o.recover(base, [m]).view(np.uint32), o.apply_quantized(base, out, 3).view(np.uint32)):
+            return False
+        # the threaded timing mode writes the same bytes and states
+        if o.compress_mt(base, cur, 3, 3).tobytes() != s.tobytes():
+            return False
+        if not np.array_equal(o.recover_mt(base, [s, s], 3).view(np.uint32), out.view(np.uint32)):
             return False
         return True
     except AssertionError:

@@ -439,3 +439,109 @@ def test_ratio_ranges_on_synthetic_deltas(oracle):
         payload_bits = int(np.frombuffer(s[40:48].tobytes(), "<u8")[0])
         assert payload_bits / (32 * n) < limit
         assert payload_bits <= n * nbits
+
+
+# ---------------------------------------------------------------- helpers the GPU parity tests lean on
+
+
+def _helper_cases():
+    rng = np.random.default_rng(61)
+    cases = []
+    for n, nbits in ((1, 1), (5, 3), (4097, 3), (3 * 4096 + 77, 8), (70001, 1), (20000, 3)):
+        base, cur = _random_case(rng, n)
+        cases.append((base, cur, nbits))
+    # a -0.0 base under an unchanged element, and deltas over a wide range of exponents (fields above 127 too)
+    n = 9000
+    base = rng.normal(0, 1.0, n).astype(np.float32)
+    base[:7] = f32([0x80000000] * 7)
+    cur = (base + (rng.normal(0, 1, n) * np.exp2(rng.integers(-40, 20, n))).astype(np.float32)).astype(np.float32)
+    cur[:7] = base[:7]
+    cases.append((base, cur, 3))
+    cases.append((base, cur, 8))
+    return cases
+
+
+def test_apply_quantized_is_recover_of_compress(oracle):
+    # Algorithm 1 step 7 computed directly must be what decoding the stream and adding gives, bit for bit.
+    for base, cur, nbits in _helper_cases():
+        direct = oracle.apply_quantized(base, cur, nbits)
+        via_stream = oracle.recover(base, [oracle.compress(base, cur, nbits)])
+        assert np.array_equal(direct.view(np.uint32), via_stream.view(np.uint32))
+    base, cur, nbits = _helper_cases()[-2]
+    assert oracle.apply_quantized(base, cur, nbits)[:7].view(np.uint32).tolist() == [0] * 7  # -0 + (+0) = +0
+
+
+def test_compress_chunks_are_slices_of_the_whole_stream(oracle):
+    for base, cur, nbits in _helper_cases():
+        n = base.size
+        s = oracle.compress(base, cur, nbits)
+        nchunks = (n + 4095) // 4096
+        nsym = int(np.frombuffer(s[16:20].tobytes(), "<u4")[0])
+        ci = 64 + 16 * nsym
+        li = ci + 8 * (nchunks + 1)
+        po = int(np.frombuffer(s[56:64].tobytes(), "<u8")[0])
+        chunk_off = np.frombuffer(s[ci:li].tobytes(), "<u8")
+        lane_bits = np.frombuffer(s[li:li + 64 * nchunks].tobytes(), "<u2").reshape(nchunks, 32)
+        ids = list(range(nchunks))[::-1]  # every chunk, in another order than the stream's
+        olane, opay = oracle.compress_chunks(base, cur, nbits, ids)
+        for k, c in enumerate(ids):
+            assert np.array_equal(olane[k], lane_bits[c])
+            assert opay[k].tobytes() == s[po + int(chunk_off[c]): po + int(chunk_off[c + 1])].tobytes()
+
+
+@pytest.mark.parametrize("threads", [1, 2, 5])
+def test_threaded_mode_gives_the_same_bytes(oracle, threads):
+    rng = np.random.default_rng(71)
+    for n, nbits in ((0, 3), (1, 2), (4096, 4), (9 * 4096 + 123, 5), (70001, 8)):
+        base, cur = _random_case(rng, n)
+        s = oracle.compress(base, cur, nbits)
+        assert oracle.compress(base, cur, nbits, threads=threads).tobytes() == s.tobytes()
+        want = oracle.recover(base, [s, s, s])
+        got = oracle.recover(base, [s, s, s], threads=threads)
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    base = np.linspace(-1, 1, 10000).astype(np.float32)  # a single used symbol: no payload
+    s = oracle.compress(base, base, 4, threads=threads)
+    assert s.tobytes() == oracle.compress(base, base, 4).tobytes()
+    assert np.array_equal(oracle.recover(base, [s], threads=threads).view(np.uint32), (base + np.float32(0)).view(np.uint32))
+
+
+# ---------------------------------------------------------------- checkpoint merging (Section 3.2)
+
+
+def test_merge_of_one_stream_over_a_zero_base_is_that_stream(oracle):
+    # With base = 0 the recovered state is the quantized delta itself; every kept bucket then holds a single value,
+    # its own representative, so quantizing again changes nothing and the merged stream is the stream, byte for byte.
+    rng = np.random.default_rng(81)
+    for n, nbits in ((10, 2), (5000, 3), (3 * 4096 + 9, 5)):
+        cur = rng.laplace(0, 1e-3, n).astype(np.float32)
+        base = np.zeros(n, np.float32)
+        s = oracle.compress(base, cur, nbits)
+        assert oracle.merge(base, [s], nbits).tobytes() == s.tobytes()
+
+
+def test_merge_is_compress_of_the_recovered_state(oracle):
+    rng = np.random.default_rng(82)
+    n = 3 * 4096 + 501
+    u0 = rng.normal(0, 0.05, n).astype(np.float32)
+    u, tracked, streams = u0.copy(), u0.copy(), []
+    for t in range(4):
+        u = (u + rng.normal(0, 1e-3, n).astype(np.float32)).astype(np.float32)
+        s = oracle.compress(tracked, u, 3)
+        streams.append(s)
+        tracked = oracle.recover(tracked, [s])
+    for k in (1, 2, 4):
+        m = oracle.merge(u0, streams[:k], 4)
+        state_k = oracle.recover(u0, streams[:k])
+        assert m.tobytes() == oracle.compress(u0, state_k, 4).tobytes()
+        # the super-step checkpoint quantizes a second time: close to the state of the k streams, within the
+        # error bound of exponent quantization (half a binade of each kept delta), not identical to it
+        back = oracle.recover(u0, [m])
+        d = (state_k - u0).astype(np.float32)
+        t4 = oracle.table(u0, state_k, 4)
+        sym = oracle.symbols(u0, state_k, 4)
+        kept = sym > 0
+        e = np.floor(np.log2(np.abs(d[kept])))
+        assert np.all(np.abs((back - u0)[kept].astype(np.float64) - d[kept]) < 2.0 ** (e - 1) + 2.0 ** -24 * np.abs(u0[kept]) * 2)
+        assert np.array_equal(back.view(np.uint32), (u0 + t4["rep"][sym]).view(np.uint32))
+    with pytest.raises(oracle.OracleError):
+        oracle.merge(u0[:-1], streams[:1], 4)  # element count mismatch
