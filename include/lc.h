@@ -9,7 +9,9 @@
  *
  * Conventions for every call
  *  - Pointers marked DEVICE are CUDA device pointers owned by the caller; pointers marked HOST are
- *    ordinary host pointers. The library allocates no memory and keeps no state between calls.
+ *    ordinary host pointers. The library allocates no memory. It keeps no state between calls except
+ *    launch parameters that it looks up once per device (SM count, occupancy, shared-memory attributes
+ *    of its kernels), and, for lc_compress_noalloc only, the built-in scratch array described there.
  *  - Work is enqueued on the CUDA stream `cs` (0 = the default stream) and, unless stated, the call
  *    returns without waiting for it. Buffers must stay valid until that work has finished.
  *  - Return value: LC_OK (0) or a negative LC_ERR_* code. Errors that only the device can see
@@ -63,7 +65,10 @@ const char* lc_strerror(int code);
  * because a Huffman code never uses more bits in total than the fixed nbits-bit code. */
 uint64_t lc_stream_bound(uint64_t n, int nbits);
 
-/* Bytes of DEVICE scratch lc_compress and lc_recover need for vectors of up to n elements. */
+/* Bytes of DEVICE scratch lc_compress and lc_recover need for vectors of up to n elements: the control block
+ * (status word, bucket statistics of Section 3.1.1, per-bucket code table), one descriptor per chunk for the
+ * scan that places the chunks (format section 3.3), and one byte per element for the bucket keys that the
+ * statistics pass hands to the encode pass. */
 uint64_t lc_workspace_bytes(uint64_t n);
 
 /*
@@ -103,13 +108,20 @@ int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbit
                        lc_cuda_stream_t cs);
 
 /*
- * lc_compress with per-kernel timing, for profiling: same arguments and result as lc_compress, but the
- * call records CUDA events around its three kernels on `cs`, waits for them, and stores the elapsed
- * milliseconds in kernel_ms (HOST float[3]: statistics pass, table pass, encode pass).
+ * lc_compress / lc_compress_update with options (the same passages; `options` only changes how the work is
+ * scheduled, never a byte of the result).
+ * tracked_out   NULL for lc_compress's behaviour, else as for lc_compress_update.
+ * options       0, or LC_OPT_NO_DEVICE_WAIT: the byte offsets of the chunks (format section 3.3) come from a
+ *               sizes pass and a one-CTA prefix-sum kernel instead of the decoupled look-back between running
+ *               CTAs of the encode pass. No kernel of the call then ever waits for another CTA, so
+ *               LC_ERR_TIMEOUT cannot occur; the price is one more pass over the one-byte key plane.
+ *               For deployments where a device-side spin, however bounded, is not acceptable.
+ * Any other bit in `options` returns LC_ERR_ARG.
  */
-int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
-                      uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs,
-                      float* kernel_ms);
+#define LC_OPT_NO_DEVICE_WAIT 1u
+int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                    uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
+                    uint32_t options, lc_cuda_stream_t cs);
 
 /*
  * Recovery pass (Algorithm 1 step 7 applied k times; u_t = u_0 + sum_i quantized delta_i).
@@ -134,11 +146,13 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs);
 int lc_last_status(const void* workspace, lc_cuda_stream_t cs);
 
 /*
- * Host-buffer variants: the same two passes for callers whose state lives in host memory (pinned
- * memory makes the copies asynchronous). Every transfer is part of the call: base, cur -> device,
- * stream -> host for compress; base, streams -> device, out -> host for recover. The device memory
- * comes from `arena` (DEVICE, 256-byte aligned, arena_bytes >= lc_host_arena_bytes()); the calls wait
+ * Host-buffer variants: the same two passes (Algorithm 1 steps 4-6 and step 7) for callers whose state lives
+ * in host memory (pinned memory makes the copies asynchronous). Every transfer is part of the call: base,
+ * cur -> device, stream -> host for compress; base, streams -> device, out -> host for recover. The device
+ * memory comes from `arena` (DEVICE, 256-byte aligned, arena_bytes >= lc_host_arena_bytes()); the calls wait
  * for `cs` before returning and return the device status as well.
+ * lc_host_arena_bytes: the workspace plus device copies of everything a call moves (two vectors and a
+ * worst-case stream for compress; one vector and k worst-case streams for recover), whichever is larger.
  */
 uint64_t lc_host_arena_bytes(uint64_t n, int nbits, int k);
 
@@ -152,17 +166,6 @@ int lc_compress_host(const float* base_host, const float* cur_host, uint64_t n, 
 int lc_recover_host(const float* base_host, const void* const* streams_host,
                     const uint64_t* stream_bytes, int k, uint64_t n, float* out_host, void* arena,
                     uint64_t arena_bytes, lc_cuda_stream_t cs);
-
-/*
- * Stage dumps for parity tests: results of the statistics and table kernels of the last lc_compress
- * that used `workspace`. All outputs HOST. Waits for `cs`.
- *   count[512], mmin[512], mmax[512]: bucket statistics by key = 256*sign + exponent field (empty
- *   bucket: mmin 0x7FFFFF, mmax 0).
- *   len[512], code[512]: code length and canonical code of the symbol each key maps to.
- */
-int lc_debug_bins(const void* workspace, uint64_t* count, uint32_t* mmin, uint32_t* mmax,
-                  lc_cuda_stream_t cs);
-int lc_debug_codes(const void* workspace, uint32_t* len, uint64_t* code, lc_cuda_stream_t cs);
 
 /*
  * Compress pass without a caller-supplied workspace. (No counterpart in the paper: this is a
@@ -179,11 +182,16 @@ int lc_debug_codes(const void* workspace, uint32_t* len, uint64_t* code, lc_cuda
  *    16-byte aligned); the stream written is byte-identical to lc_compress's.
  *  - The call waits for `cs` and returns the device status as well (LC_ERR_NONFINITE, LC_ERR_TIMEOUT).
  *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
- *    that device current). Make that first call outside any CUDA stream capture.
+ *    that device current). With CUDA's default lazy module loading that look-up is also what loads the
+ *    part of the library that holds the array, i.e. the moment the driver reserves the array's device
+ *    memory, and it may synchronise the device. A caller whose pool is about to take the whole device
+ *    must therefore make that first call at start-up, before the pool grows (n = 0 is enough: it does
+ *    the look-up and writes a header-only stream), or run with CUDA_MODULE_LOADING=EAGER. Make it
+ *    outside any CUDA stream capture. Later calls allocate nothing.
  *  - Every call on a device shares the one array, which keeps the previous call's contents (the call
  *    clears what must start at zero). Two calls that overlap on the same GPU race: do not issue them
  *    from different streams or threads at the same time.
- *  - The array (about 4.8 MB) stays resident on every GPU that loads the library, until exit.
+ *  - The array (about 4.2 MB) stays resident on every GPU that loads the library, until exit.
  */
 #define LC_NOALLOC_MAX_N 4194304ull
 int lc_compress_noalloc(const float* base, const float* cur, uint64_t n, int nbits, void* stream,

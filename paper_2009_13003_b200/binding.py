@@ -18,7 +18,7 @@ MAX_CHAIN = 8
 
 SYMBOLS = (
     "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_update", "lc_compress_timed",
-    "lc_recover",
+    "lc_recover", "lc_compress_opt", "lc_debug_compress_wait",
     "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
     "lc_debug_bins", "lc_debug_codes", "lc_compress_noalloc",
 )
@@ -64,6 +64,8 @@ def lib():
     L.lc_workspace_bytes.restype = u64
     L.lc_compress.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp]
     L.lc_compress_update.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
+    L.lc_compress_opt.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, C.c_uint32, vp]
+    L.lc_debug_compress_wait.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, C.c_uint32, C.c_uint32, vp]
     L.lc_compress_timed.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, C.POINTER(C.c_float)]
     L.lc_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
     L.lc_stream_info.argtypes = [vp, C.POINTER(LCInfo), vp]
@@ -130,6 +132,26 @@ def compress_update_async(base, cur, nbits, stream, tracked_out, workspace):
                                   stream.numel(), tracked_out.data_ptr(), workspace.data_ptr(), workspace.numel(),
                                   _cs(base.device))
     _check(rc, "lc_compress_update")
+
+
+OPT_NO_DEVICE_WAIT = 1
+
+
+def compress_opt_async(base, cur, nbits, stream, workspace, options, tracked_out=None):
+    """Enqueues lc_compress_opt (``options``: 0 or OPT_NO_DEVICE_WAIT; ``tracked_out`` as for lc_compress_update)."""
+    _f32_cuda(base, "base"), _f32_cuda(cur, "cur")
+    rc = lib().lc_compress_opt(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(), stream.numel(),
+                               None if tracked_out is None else tracked_out.data_ptr(), workspace.data_ptr(),
+                               workspace.numel(), options, _cs(base.device))
+    _check(rc, "lc_compress_opt")
+
+
+def debug_compress_wait(base, cur, nbits, stream, workspace, spin_limit, first_ticket):
+    """lc_debug_compress_wait: lc_compress with the look-back's poll limit and first tile number given."""
+    rc = lib().lc_debug_compress_wait(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(),
+                                      stream.numel(), workspace.data_ptr(), workspace.numel(), spin_limit,
+                                      first_ticket, _cs(base.device))
+    _check(rc, "lc_debug_compress_wait")
 
 
 def compress_timed(base, cur, nbits, stream, workspace):

@@ -2,6 +2,7 @@
 #include <string.h>
 
 #include "lc_common.cuh"
+#include "../../include/lc_debug.h"
 
 using namespace lc;
 
@@ -26,7 +27,8 @@ Carved carve(void* workspace, const WorkspaceLayout& W) {
 
 // lc_compress and lc_compress_update: argument checks, then memset + three kernels on `cs`.
 int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, void* stream, uint64_t stream_capacity,
-                  float* tracked_out, void* workspace, uint64_t workspace_bytes, cudaStream_t cs) {
+                  float* tracked_out, void* workspace, uint64_t workspace_bytes, const EncodeOptions& opt,
+                  cudaStream_t cs) {
   if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
   if (!stream || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
   if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
@@ -40,9 +42,16 @@ int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, vo
   if (e != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), tracked_out, cs)) !=
-      cudaSuccess)
+  if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), tracked_out, opt,
+                         cs)) != cudaSuccess)
     return LC_ERR_CUDA;
+  return LC_OK;
+}
+
+int check_tracked_out(const float* cur, uint64_t n, float*& tracked_out) {
+  if (n > 0 && (!tracked_out || !aligned(tracked_out, 16))) return LC_ERR_ARG;
+  if (n > 0 && tracked_out == cur) return LC_ERR_ARG;  // cur is read after parts of tracked_out are written
+  if (n == 0) tracked_out = nullptr;
   return LC_OK;
 }
 
@@ -76,16 +85,39 @@ uint64_t lc_workspace_bytes(uint64_t n) { return workspace_layout(n).total; }
 
 int lc_compress(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                 uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
-  return compress_impl(base, cur, n, nbits, stream, stream_capacity, nullptr, workspace, workspace_bytes, cs);
+  return compress_impl(base, cur, n, nbits, stream, stream_capacity, nullptr, workspace, workspace_bytes,
+                       EncodeOptions(), cs);
 }
 
 int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                        uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
                        lc_cuda_stream_t cs) {
-  if (n > 0 && (!tracked_out || !aligned(tracked_out, 16))) return LC_ERR_ARG;
-  if (n > 0 && tracked_out == cur) return LC_ERR_ARG;  // cur is read after parts of tracked_out are written
-  if (n == 0) tracked_out = nullptr;
-  return compress_impl(base, cur, n, nbits, stream, stream_capacity, tracked_out, workspace, workspace_bytes, cs);
+  const int rc = check_tracked_out(cur, n, tracked_out);
+  if (rc != LC_OK) return rc;
+  return compress_impl(base, cur, n, nbits, stream, stream_capacity, tracked_out, workspace, workspace_bytes,
+                       EncodeOptions(), cs);
+}
+
+int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                    uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
+                    uint32_t options, lc_cuda_stream_t cs) {
+  if (options & ~(uint32_t)LC_OPT_NO_DEVICE_WAIT) return LC_ERR_ARG;
+  if (tracked_out) {
+    const int rc = check_tracked_out(cur, n, tracked_out);
+    if (rc != LC_OK) return rc;
+  }
+  EncodeOptions opt;
+  opt.two_pass_scan = (options & LC_OPT_NO_DEVICE_WAIT) != 0;
+  return compress_impl(base, cur, n, nbits, stream, stream_capacity, tracked_out, workspace, workspace_bytes, opt, cs);
+}
+
+int lc_debug_compress_wait(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                           uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, uint32_t spin_limit,
+                           uint32_t first_ticket, lc_cuda_stream_t cs) {
+  EncodeOptions opt;
+  opt.spin_limit = spin_limit;
+  opt.ticket_bias = first_ticket;
+  return compress_impl(base, cur, n, nbits, stream, stream_capacity, nullptr, workspace, workspace_bytes, opt, cs);
 }
 
 int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
@@ -108,7 +140,7 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
   ok = ok && cudaEventRecord(ev[1], cs) == cudaSuccess;
   ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[2], cs) == cudaSuccess;
-  ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, cs) == cudaSuccess;
+  ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[3], cs) == cudaSuccess;
   ok = ok && cudaEventSynchronize(ev[3]) == cudaSuccess;
   for (int i = 0; ok && i < 3; ++i) ok = cudaEventElapsedTime(&kernel_ms[i], ev[i], ev[i + 1]) == cudaSuccess;

@@ -99,13 +99,32 @@ __host__ __device__ inline WorkspaceLayout workspace_layout(uint64_t n) {
 // ---- device helpers ----------------------------------------------------------------------------
 __device__ inline void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
 
+// ---- per-device launch parameters ---------------------------------------------------------------------
+// Occupancy figures, SM counts and the "attributes are set" marks that the launchers cache are properties of a
+// device (cudaFuncSetAttribute applies to the current device only), so every such cache is an array indexed by
+// the device ordinal. Returns -1 if the ordinal cannot be had or is beyond the arrays.
+constexpr int kMaxDevices = 64;
+inline int current_device_index() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
+// How the encode pass finds the byte offset of a tile of chunks, and the limits of its bounded wait.
+struct EncodeOptions {
+  bool two_pass_scan = false;     // offsets from a sizes pass and a one-CTA scan: no CTA ever waits for another
+  uint32_t spin_limit = 1u << 20; // polls of the look-back before it gives up with LC_ERR_TIMEOUT
+  uint32_t ticket_bias = 0;       // added to every tile ticket (test aid: with 1, tile 0 is never coded)
+};
+
 // ---- launchers (each defined next to its kernel) ---------------------------------------------------
 cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
                          cudaStream_t cs);
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, cudaStream_t cs);
 // tracked_out: nullptr, or where to write base + quantized delta (may be base itself)
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
-                          const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, cudaStream_t cs);
+                          const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, const EncodeOptions& opt,
+                          cudaStream_t cs);
 
 struct DecodeStreams {
   const uint8_t* ptr[4];

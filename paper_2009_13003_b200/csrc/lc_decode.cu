@@ -29,10 +29,12 @@
 //
 // Bound: HBM at k = 1 (8 bytes per element + the stream); at k = 4 the integer work per symbol is
 // the limit.
-#include "lc_common.cuh"
+#include "lc_decode_bits.cuh"
 
 namespace lc {
 namespace {
+
+using namespace dec;
 
 constexpr int kDecMaxThreads = 512;
 constexpr int kL1Bits = 6;
@@ -41,7 +43,6 @@ constexpr int kSubBitsMax = 6;                     // second level: the next 6 b
 constexpr int kSubBitsMin = 4;
 constexpr int kL2Bits = kL1Bits + kSubBitsMax;     // longest code the two table levels resolve
 constexpr uint32_t kLongCode = 0xFFFFFFFFu;
-constexpr uint32_t kOverrunBytes = 512;  // padding behind the last staging area (see LaneBits::refill)
 static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill guarantee");
 
 // The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory.
@@ -71,14 +72,6 @@ struct alignas(16) StreamState {
 };
 
 static_assert(sizeof(StreamState) % 16 == 0, "the staging areas behind the tables take 16-byte accesses");
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ uint64_t load_le(const uint8_t* p, int bytes) {
-  uint64_t v = 0;
-  for (int b = 0; b < bytes; ++b) v |= (uint64_t)p[b] << (8 * b);
-  return v;
-}
 
 // Canonical decode of the top `width` bits `idx`: (index into sorted_rep, length) or length 0 if the code
 // is longer than `width`.
@@ -261,24 +254,6 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   return 0;
 }
 
-// ---- shared-memory access by 32-bit shared address (keeps the hot loop free of generic addressing)
-__device__ __forceinline__ uint32_t lds_u32(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
-// 16-byte load of base; volatile so that it stays where it is written (early in the loop body). A plain cached
-// load: measured a few percent faster than the streaming forms with one stream, the same with four.
-__device__ __forceinline__ float4 ldg_stream_v4(const float* p) {
-  float4 v;
-  asm volatile("ld.global.nc.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
-  return v;
-}
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 // Two-level table lookup of the code at the top of `hi`: {representative, length}, length kLongCode if
 // the tables do not resolve it. `l1lane` = shared address of this lane's copy of first-level entry 0.
 // The first-level entry of a prefix that belongs to longer codes holds the shared address of the
@@ -304,14 +279,6 @@ __device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane, uint3
   return ent;
 }
 
-// Where a chunk's words are read from.
-struct Source {
-  const uint32_t* g;  // chunk words in global memory
-  uint32_t nw;        // words in the chunk
-  uint32_t sbase;     // staged: shared address of the chunk's first word
-  uint32_t slim;      // staged: shared address of the last readable word (zero slack after the chunk)
-};
-
 // Table-free canonical decode of the code that starts at bit `bitpos` of a chunk in global memory
 // (the slow path for ragged or oversized chunks): {representative, length}.
 __device__ __noinline__ uint2 decode_any(const StreamState& S, const uint32_t* g, uint32_t nw, uint32_t bitpos,
@@ -330,79 +297,6 @@ __device__ __noinline__ uint2 decode_any(const StreamState& S, const uint32_t* g
   set_status(status, LC_ERR_FORMAT);  // no code matches: damaged payload
   return make_uint2(0u, S.max_len);
 }
-
-// A lane's read state in one stream: `cnt` valid bits at the top of hi:lo (the bits below are zero).
-// STAGED: the chunk's words are in the warp's staging area and `next` is the shared address of the next
-// word to load. Otherwise (a chunk too large to stage) they are read from global memory and `next` is a
-// word index.
-template <bool STAGED>
-struct LaneBits {
-  uint32_t hi, lo;
-  int cnt;
-  uint32_t next;
-
-  // word `idx` of the chunk, 0 beyond its end
-  __device__ __forceinline__ static uint32_t word(const Source& W, uint32_t idx) {
-    if (STAGED) return lds_u32(min(W.sbase + idx * 4u, W.slim));
-    return idx < W.nw ? __ldg(W.g + idx) : 0u;
-  }
-  __device__ __forceinline__ uint32_t bitpos(const Source& W) const {
-    return (STAGED ? (next - W.sbase) * 8u : next * 32u) - (uint32_t)cnt;
-  }
-  __device__ __forceinline__ void seek(const Source& W, uint32_t pos) {
-    const uint32_t idx = pos >> 5, sh = pos & 31;
-    const uint32_t w0 = word(W, idx), w1 = word(W, idx + 1);
-    hi = __funnelshift_l(w1, w0, sh);
-    lo = w1 << sh;
-    cnt = 64 - (int)sh;
-    next = STAGED ? min(W.sbase + (idx + 2) * 4u, W.slim) : idx + 2;
-  }
-  // Tops the buffer up with one word if 32 bits or fewer are left; afterwards cnt >= 33. All predicated.
-  // STAGED: the load is not clamped: between two seeks (which do clamp) `next` moves by at most 64 words,
-  // and the kernel's shared memory ends with kOverrunBytes of padding, so a damaged stream can make a lane
-  // read stale shared memory but never leave the allocation.
-  __device__ __forceinline__ void refill(const Source& W) {
-    if (STAGED) {
-      asm volatile(
-          "{\n\t"
-          ".reg .pred q;\n\t"
-          ".reg .u32 w, t;\n\t"
-          "setp.le.s32 q, %2, 32;\n\t"
-          "@q ld.shared.u32 w, [%3];\n\t"
-          "@q shf.r.clamp.b32 t, w, 0, %2;\n\t"   // high word of (w:0) >> cnt, i.e. w >> cnt (0 when cnt == 32)
-          "@q or.b32 %0, %0, t;\n\t"
-          "@q shf.r.clamp.b32 %1, 0, w, %2;\n\t"  // low word of (w:0) >> cnt; lo was 0 because cnt <= 32
-          "@q add.s32 %2, %2, 32;\n\t"
-          "@q add.u32 %3, %3, 4;\n\t"
-          "}"
-          : "+r"(hi), "+r"(lo), "+r"(cnt), "+r"(next));
-    } else {
-      asm volatile(
-          "{\n\t"
-          ".reg .pred q, r;\n\t"
-          ".reg .u32 w, t;\n\t"
-          ".reg .u64 a;\n\t"
-          "setp.le.s32 q, %2, 32;\n\t"
-          "setp.lt.and.u32 r, %3, %5, q;\n\t"     // words beyond the chunk read as 0
-          "mov.u32 w, 0;\n\t"
-          "mad.wide.u32 a, %3, 4, %4;\n\t"
-          "@r ld.global.nc.u32 w, [a];\n\t"
-          "@q shf.r.clamp.b32 t, w, 0, %2;\n\t"
-          "@q or.b32 %0, %0, t;\n\t"
-          "@q shf.r.clamp.b32 %1, 0, w, %2;\n\t"
-          "@q add.s32 %2, %2, 32;\n\t"
-          "@q add.u32 %3, %3, 1;\n\t"
-          "}"
-          : "+r"(hi), "+r"(lo), "+r"(cnt), "+r"(next)
-          : "l"(W.g), "r"(W.nw));
-    }
-  }
-  __device__ __forceinline__ void consume(uint32_t len) {
-    hi = __funnelshift_l(lo, hi, len);
-    lo <<= len;
-    cnt -= (int)len;
-  }
-};
 
 // Code the tables did not resolve: canonical search on a 64-bit window read from the chunk, then re-seat
 // the lane's bit buffer behind the code. Returns the representative.
@@ -501,11 +395,6 @@ __device__ __noinline__ void decode_chunk_global(const StreamState* S, GlobalChu
       float x = base[i];
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        const uint32_t wi = pos[s] >> 5, sh = pos[s] & 31;
-        const uint32_t w0 = wi < G.nw[s] ? __ldg(G.g[s] + wi) : 0u;
-        const uint32_t w1 = wi + 1 < G.nw[s] ? __ldg(G.g[s] + wi + 1) : 0u;
-        const uint32_t peek = __funnelshift_l(w1, w0, sh);
-        (void)peek;
         const uint2 ent = decode_any(S[s], G.g[s], G.nw[s], pos[s], status);
         x = __fadd_rn(x, __uint_as_float(ent.x));
         pos[s] += ent.y;
@@ -610,24 +499,24 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
   }
 }
 
-constexpr uint32_t kSmemPerSm = 227 * 1024;  // usable shared memory of one CTA on sm_100
-
 template <int KS>
 cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, uint64_t n, float* out,
                              int32_t* status, cudaStream_t cs) {
-  static int sms = 0;
+  static int sms_of[kMaxDevices] = {};  // by device ordinal; non-zero once the kernel's attributes are set there
   constexpr uint32_t kTables = kTableBytes + KS * (2 * kTableBytes + sizeof(StreamState));
   constexpr uint32_t kMaxDyn = kSmemPerSm - 1024 - kOverrunBytes;  // room for static __shared__ and the padding
-  if (sms == 0) {
-    int dev = 0, v = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+  const int dev = current_device_index();
+  if (dev < 0) return cudaErrorInvalidDevice;
+  if (sms_of[dev] == 0) {
+    int v = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     e = cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(kMaxDyn + kOverrunBytes));
     if (e != cudaSuccess) return e;
-    sms = v;
+    sms_of[dev] = v;
   }
+  const int sms = sms_of[dev];
   const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
   // Staging per warp and stream: 1.03 x the largest average chunk of the streams (from the buffer sizes,
   // which bound the payload). Among CTAs of 16, 12 and 8 warps, take the shape that puts most warps on an

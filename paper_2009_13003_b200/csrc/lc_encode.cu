@@ -21,8 +21,12 @@
 // The loop is software-pipelined: D and E of a tile run after A and B of the CTA's next tile (whose C follows
 // once E has freed the image area), and D is done by whichever warp finishes coding first (see the loop). Tiles are handed out by an atomic ticket, so
 // every tile a CTA waits for in D has already been started by a running CTA, and coding never waits for
-// anything. The wait is bounded all the same: after kSpinLimit polls the CTA records LC_ERR_TIMEOUT, marks
+// anything. The wait is bounded all the same: after `spin_limit` polls the CTA records LC_ERR_TIMEOUT, marks
 // its tile aborted (successors see that at once and abort too) and moves on.
+// A caller that wants no device-side wait at all selects the two-pass scan (EncodeOptions::two_pass_scan):
+// encode_sizes_kernel computes every chunk's size, encode_scan_kernel (one CTA) turns the sizes into the chunk
+// index, and this kernel takes its offsets from there instead of looking back. Same bytes, one more pass over
+// the key plane.
 //
 // Rare cases take a compact two-pass path (lengths, then bits ORed in place): the ragged last chunk,
 // codes longer than 32 bits, a lane or chunk that outgrows its shared-memory area, and vectors with an
@@ -39,7 +43,6 @@ constexpr int kEncThreads = kEncWarps * 32;
 // 48 KB of dynamic shared memory per CTA (four CTAs per SM), split evenly between the warps that work:
 // all 8 while an average chunk fits half of a 6 KB share (column matrix + chunk image), else 4, 2 or 1.
 constexpr uint32_t kEncSmem = 48 * 1024;
-constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr int kUpdRows = 4;  // rows of base in flight per warp in the kernel that also writes the tracked state
 constexpr uint32_t kUpdSmem = kEncWarps * kUpdRows * 512;  // its ring, behind the kEncSmem bytes of coding areas
 constexpr int kLookBack = 8;  // look-back sub-windows of 32 tile descriptors read per round
@@ -163,7 +166,7 @@ template <bool UPDATE>
 __global__ void __launch_bounds__(kEncThreads, UPDATE ? 3 : 4)
 encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles, const uint8_t* __restrict__ plane,
               const float* base, const float* __restrict__ cur, uint64_t n, uint8_t* __restrict__ stream,
-              float* tracked_out) {
+              float* tracked_out, uint32_t spin_limit, uint32_t ticket_bias, uint32_t two_pass_scan) {
   extern __shared__ __align__(16) uint32_t s_dyn[];
   __shared__ Tables tb;
   __shared__ uint32_t s_chunk_bytes[2][kEncWarps];  // [half][warp]: the pending tile and the one being coded
@@ -174,9 +177,14 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
   __shared__ uint32_t s_arrived[2];  // warps that have coded their chunk of the tile in this half
   __shared__ uint32_t s_rep[UPDATE ? 256 : 1];  // UPDATE: representative (bit pattern) by plane byte
 
-  if (ctl->status != 0) return;  // the table pass rejected the vector
-
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // The table pass may have rejected the vector, or another CTA may already have given up waiting: leave, all
+  // threads together (one thread reads the word; a thread-by-thread test could split the CTA if the word changed
+  // in between, and the warps that stayed would wait at barriers for the ones that left).
+  if (tid == 0) s_abort = ctl->status;
+  __syncthreads();
+  if (s_abort != 0) return;
+  __syncthreads();  // everybody has read s_abort before thread 0 reuses it below
   for (uint32_t b = tid; b < 256; b += kEncThreads) {
     const EncEntry e = ctl->enc[((b & 1u) << 8) | (b >> 1)];
     tb.full[b] = make_uint2(e.code_lo, e.len);
@@ -249,7 +257,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
   uint32_t p_tile = 0, p_buf = 0;
 
   if (tid == 0) {
-    s_tile = atomicAdd(&ctl->ticket, 1u);
+    s_tile = atomicAdd(&ctl->ticket, 1u) + ticket_bias;
     s_abort = 0;
     s_arrived[0] = s_arrived[1] = 0;
   }
@@ -360,7 +368,10 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     if (p_have && arrival == 0) {
       unsigned long long part = 0;  // this lane's share of the sum
       bool abort = false;
-      if (p_tile > 0) {
+      if (two_pass_scan) {
+        // the chunk index is already there (encode_scan_kernel): the tile starts where its first chunk starts
+        if (lane == 0) part = chunk_index[(uint64_t)p_tile * active];
+      } else if (p_tile > 0) {
         long long look = (long long)p_tile - 1;
         uint32_t spins = 0;
         bool done = false;
@@ -394,7 +405,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
             }
           }
           if (retry) {
-            if (++spins > kSpinLimit) abort = true;
+            if (++spins > spin_limit) abort = true;
             else __nanosleep(40);
           }
         }
@@ -410,7 +421,8 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
           unsigned long long p_tile_bytes = 0;
 #pragma unroll
           for (int w = 0; w < (int)kEncWarps; ++w) p_tile_bytes += s_chunk_bytes[p_buf][w];
-          if (p_tile > 0) st_tile(&tiles[p_tile], (kTilePrefix << kTileFlagShift) | (part + p_tile_bytes));
+          if (p_tile > 0 && !two_pass_scan)
+            st_tile(&tiles[p_tile], (kTilePrefix << kTileFlagShift) | (part + p_tile_bytes));
           s_abort = 0;
           s_tile_base = part;
           s_tile_end = part + p_tile_bytes;
@@ -420,7 +432,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     __syncthreads();  // all chunk sizes of the new tile, and the pending tile's offset, are known
     if (tid == 0) {
       s_arrived[p_buf] = 0;  // the other half's counter, for the next iteration
-      if (have) {
+      if (have && !two_pass_scan) {
         unsigned long long tile_bytes = 0;
 #pragma unroll
         for (int w = 0; w < (int)kEncWarps; ++w) tile_bytes += s_chunk_bytes[buf][w];
@@ -498,7 +510,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
     if (!have) break;
     // The next ticket is taken now, so that the round trip overlaps the rest of this iteration. (Taking it
     // earlier would only make the tile look late to its successors: its size cannot appear before it is coded.)
-    if (tid == 0) s_tile = atomicAdd(&ctl->ticket, 1u);
+    if (tid == 0) s_tile = atomicAdd(&ctl->ticket, 1u) + ticket_bias;
     __syncwarp();  // the warp's image area is free again
 
     // ---- C: assemble the new tile's chunk image in shared memory
@@ -528,32 +540,100 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
   }
 }
 
+// ---- two-pass scan: chunk sizes, then their exclusive prefix sum, with no CTA waiting for another ----------
+
+constexpr int kScanThreads = 1024;
+
+// Size in bytes of every chunk (format section 3.3: the chunk's bits rounded up to 16 bytes), one warp per chunk,
+// into sizes[c].
+__global__ void __launch_bounds__(kEncThreads)
+encode_sizes_kernel(const Control* __restrict__ ctl, unsigned long long* __restrict__ sizes,
+                    const uint8_t* __restrict__ plane, const float* base, const float* __restrict__ cur, uint64_t n,
+                    uint64_t nchunks) {
+  if (ctl->status != 0) return;  // nothing in this kernel writes the word: the same for every thread
+  const uint32_t lane = threadIdx.x & 31;
+  const KeySource ks{plane, base, cur, ctl->wide != 0};
+  const uint64_t warp0 = (uint64_t)blockIdx.x * kEncWarps + (threadIdx.x >> 5), nwarps = (uint64_t)gridDim.x * kEncWarps;
+  for (uint64_t c = warp0; c < nchunks; c += nwarps) {
+    uint32_t bits = chunk_slow(ctl->enc, ks, c, lane, n, nullptr, 0);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) bits += __shfl_xor_sync(0xffffffffu, bits, d);
+    if (lane == 0) sizes[c] = align_up((bits + 7) / 8, kPayloadAlign);
+  }
+}
+
+// chunk_off[c] = sum of sizes[0..c) for c = 0..nchunks, and the stream's total size into its header. One CTA:
+// each thread sums a contiguous run of chunks, the run totals are scanned in shared memory.
+__global__ void __launch_bounds__(kScanThreads)
+encode_scan_kernel(const Control* __restrict__ ctl, const unsigned long long* __restrict__ sizes, uint64_t n,
+                   uint64_t nchunks, uint8_t* __restrict__ stream) {
+  __shared__ unsigned long long run_total[kScanThreads];
+  if (ctl->status != 0) return;
+  const StreamLayout L = stream_layout(n, ctl->nsym);
+  unsigned long long* chunk_index = reinterpret_cast<unsigned long long*>(stream + L.chunk_index_off);
+  const uint64_t per = (nchunks + kScanThreads - 1) / kScanThreads;
+  const uint64_t lo = min(nchunks, per * threadIdx.x), hi = min(nchunks, lo + per);
+  unsigned long long sum = 0;
+  for (uint64_t c = lo; c < hi; ++c) sum += sizes[c];
+  run_total[threadIdx.x] = sum;
+  __syncthreads();
+  for (int d = 1; d < kScanThreads; d <<= 1) {  // inclusive scan of the run totals
+    const unsigned long long v = (int)threadIdx.x >= d ? run_total[threadIdx.x - d] : 0ull;
+    __syncthreads();
+    run_total[threadIdx.x] += v;
+    __syncthreads();
+  }
+  unsigned long long off = run_total[threadIdx.x] - sum;
+  for (uint64_t c = lo; c < hi; ++c) {
+    chunk_index[c] = off;
+    off += sizes[c];
+  }
+  if (threadIdx.x == kScanThreads - 1) {
+    chunk_index[nchunks] = run_total[kScanThreads - 1];
+    *reinterpret_cast<unsigned long long*>(stream + 48) = L.payload_off + run_total[kScanThreads - 1];
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
-                          const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, cudaStream_t cs) {
+                          const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, const EncodeOptions& opt,
+                          cudaStream_t cs) {
   const WorkspaceLayout W = workspace_layout(n);
   if (W.nchunks == 0) return cudaSuccess;
-  static int blocks_per_sm[2] = {0, 0}, sms = 0;
+  static int blocks_per_sm[kMaxDevices][2] = {}, sms[kMaxDevices] = {};  // by device ordinal
+  const int dev = current_device_index();
+  if (dev < 0) return cudaErrorInvalidDevice;
   const int v = tracked_out ? 1 : 0;
-  if (blocks_per_sm[v] == 0) {
+  if (blocks_per_sm[dev][v] == 0) {
     const void* fn = v ? reinterpret_cast<const void*>(encode_kernel<true>) : reinterpret_cast<const void*>(encode_kernel<false>);
     cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncSmem + (v ? kUpdSmem : 0));
     if (e != cudaSuccess) return e;
-    int dev = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    int nsm = 0;
+    if ((e = cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     int bps = 0;
     e = v ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, encode_kernel<true>, kEncThreads, kEncSmem + kUpdSmem)
           : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, encode_kernel<false>, kEncThreads, kEncSmem);
     if (e != cudaSuccess) return e;
-    blocks_per_sm[v] = bps > 0 ? bps : 1;
+    sms[dev] = nsm;
+    blocks_per_sm[dev][v] = bps > 0 ? bps : 1;
   }
   const uint64_t want = (W.nchunks + kEncWarps - 1) / kEncWarps;
-  const uint64_t full = (uint64_t)sms * blocks_per_sm[v];
+  const uint64_t full = (uint64_t)sms[dev] * blocks_per_sm[dev][v];
   const unsigned grid = (unsigned)(want < full ? want : full);
-  if (v) encode_kernel<true><<<grid, kEncThreads, kEncSmem + kUpdSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, tracked_out);
-  else encode_kernel<false><<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, nullptr);
+  if (opt.two_pass_scan) {
+    // tiles[] (zeroed by the caller, one entry per chunk) holds the chunk sizes in this mode
+    encode_sizes_kernel<<<grid, kEncThreads, 0, cs>>>(ctl, tiles, plane, base, cur, n, W.nchunks);
+    encode_scan_kernel<<<1, kScanThreads, 0, cs>>>(ctl, tiles, n, W.nchunks, stream);
+    if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
+  }
+  const uint32_t two = opt.two_pass_scan ? 1u : 0u;
+  if (v)
+    encode_kernel<true><<<grid, kEncThreads, kEncSmem + kUpdSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, tracked_out,
+                                                                       opt.spin_limit, opt.ticket_bias, two);
+  else
+    encode_kernel<false><<<grid, kEncThreads, kEncSmem, cs>>>(ctl, tiles, plane, base, cur, n, stream, nullptr,
+                                                              opt.spin_limit, opt.ticket_bias, two);
   return cudaGetLastError();
 }
 

@@ -23,7 +23,6 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
 // In host code the name above is only a handle; the device address has to be asked for, once per
 // device, with that device current.
-constexpr int kMaxDevices = 64;
 void* g_scratch_addr[kMaxDevices] = {};
 
 int scratch_for_current_device(void** out) {
@@ -63,7 +62,7 @@ extern "C" int lc_compress_noalloc(const float* base, const float* cur, uint64_t
   if (cudaMemsetAsync(w, 0, W.plane_off, cs) != cudaSuccess) return LC_ERR_CUDA;
   if (launch_stats(base, cur, n, ctl, plane, cs) != cudaSuccess) return LC_ERR_CUDA;
   if (launch_table(ctl, n, nbits, static_cast<uint8_t*>(stream), cs) != cudaSuccess) return LC_ERR_CUDA;
-  if (launch_encode(ctl, tiles, plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, cs) != cudaSuccess)
+  if (launch_encode(ctl, tiles, plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(), cs) != cudaSuccess)
     return LC_ERR_CUDA;
   int32_t status = 0;
   if (cudaMemcpyAsync(&status, &ctl->status, sizeof status, cudaMemcpyDeviceToHost, cs) != cudaSuccess)

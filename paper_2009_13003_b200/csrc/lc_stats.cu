@@ -162,25 +162,28 @@ cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Contro
                          cudaStream_t cs) {
   const WorkspaceLayout W = workspace_layout(n);
   if (W.nunits == 0) return cudaSuccess;
-  static int blocks_per_sm = 0, sms = 0;
-  if (blocks_per_sm == 0) {
+  static int blocks_per_sm[kMaxDevices] = {}, sms[kMaxDevices] = {};  // by device ordinal
+  const int dev = current_device_index();
+  if (dev < 0) return cudaErrorInvalidDevice;
+  if (blocks_per_sm[dev] == 0) {
     cudaError_t e = cudaFuncSetAttribute(stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmem);
     if (e != cudaSuccess) return e;
-    int dev = 0;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    int nsm = 0;
+    if ((e = cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     int bps = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, stats_kernel, kStatsThreads, kStatsSmem);
     if (e != cudaSuccess) return e;
-    blocks_per_sm = bps > 0 ? bps : 1;
+    if (bps < 1) bps = 1;
     // carve-out in percent of the SM's 228 KB: the resident CTAs' shared memory (plus 1 KB each that the system
     // reserves), rounded up
-    const int carve = (int)(((uint64_t)blocks_per_sm * (kStatsSmem + 1024) * 100 + 228 * 1024 - 1) / (228 * 1024)) + 1;
+    const int carve = (int)(((uint64_t)bps * (kStatsSmem + 1024) * 100 + 228 * 1024 - 1) / (228 * 1024)) + 1;
     e = cudaFuncSetAttribute(stats_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve < 100 ? carve : 100);
     if (e != cudaSuccess) return e;
+    sms[dev] = nsm;
+    blocks_per_sm[dev] = bps;
   }
   const uint64_t want = (W.nunits + kStatsThreads / 32 - 1) / (kStatsThreads / 32);
-  const uint64_t full = (uint64_t)sms * blocks_per_sm;
+  const uint64_t full = (uint64_t)sms[dev] * blocks_per_sm[dev];
   const unsigned grid = (unsigned)(want < full ? want : full);
   stats_kernel<<<grid, kStatsThreads, kStatsSmem, cs>>>(base, cur, n, W.nunits, ctl, plane);
   return cudaGetLastError();

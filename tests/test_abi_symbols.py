@@ -1,4 +1,5 @@
-"""The C-ABI library loads without a GPU and exports every function include/lc.h declares."""
+"""The C-ABI library loads without a GPU and exports every function the headers under include/ declare."""
+import glob
 import os
 import re
 
@@ -6,7 +7,7 @@ from conftest import ROOT
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "lc.h")).read()
+    text = "".join(open(h).read() for h in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(lc_[a-z_0-9]+)\s*\(", text)))
 
@@ -51,3 +52,17 @@ def test_host_argument_checks_need_no_device():
     assert upd(0x50000, nbits=9) == binding.ERR_ARG
     assert L.lc_compress_update(base, cur, 16, 4, stream, 8, 0x50000, ws, 1 << 20, None) == binding.ERR_CAPACITY
     assert L.lc_strerror(binding.ERR_FORMAT) == b"malformed stream"
+    # lc_compress_opt: unknown option bits are refused before anything else happens
+    assert L.lc_compress_opt(base, cur, 16, 4, stream, 1 << 20, None, ws, 1 << 20, 2, None) == binding.ERR_ARG
+    assert L.lc_compress_opt(base, cur, 16, 4, stream, 1 << 20, cur, ws, 1 << 20, 1, None) == binding.ERR_ARG
+
+
+def test_launch_parameter_caches_are_per_device():
+    # Function attributes and occupancy belong to a device: a function-scope static that caches them must be an
+    # array indexed by the device ordinal (a process may use several GPUs).
+    csrc = os.path.join(ROOT, "paper_2009_13003_b200", "csrc")
+    for path in sorted(glob.glob(os.path.join(csrc, "*.cu"))):
+        text = re.sub(r"//.*", "", open(path).read())
+        for m in re.finditer(r"^\s+static\s+(?!_|const|constexpr)[^;(]*;", text, flags=re.M):
+            decl = m.group(0)
+            assert "[kMaxDevices]" in decl, "%s: %s" % (os.path.basename(path), decl.strip())

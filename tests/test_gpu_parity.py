@@ -5,6 +5,8 @@ codebook, whole stream) and bit-exact fp32 for the recovered state (the represen
 integers on the GPU and in double on the CPU, both exact; spec tolerance 1e-6 relative is the
 fallback threshold stated in ``REL_TOL`` and checked as well).
 """
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -12,6 +14,8 @@ import torch
 pytestmark = pytest.mark.gpu
 
 REL_TOL = 1e-6
+# host threads for the oracle's chunk-parallel mode (byte-identical to its single-threaded pass, pinned on the CPU)
+ORACLE_THREADS = max(1, min(os.cpu_count() or 1, 64))
 
 
 @pytest.fixture(scope="module")
@@ -138,6 +142,28 @@ def test_sweep_distributions(lc, oracle, nbits, dist):
     cur = base + synth.sweep_delta(dist, n, DEV, 11 + nbits)
     got, _ = assert_stream_parity(lc, oracle, base, cur, nbits)
     assert_recover_parity(lc, oracle, base, [got], inplace=(nbits % 2 == 0))
+
+
+@pytest.mark.parametrize("logn", [24, 28])
+@pytest.mark.parametrize("dist", ["lognormal", "one_exp", "zero"])
+def test_sweep_at_benchmarked_sizes(lc, oracle, logn, dist):
+    # the sizes of the sweep table (2^24 fits the L2, 2^28 does not), against the oracle on all host cores
+    from paper_2009_13003_b200 import synth
+
+    n, nbits = 1 << logn, 5
+    base = synth.normal(n, 0.02, DEV, synth.SEED0 + 5)
+    if dist == "one_exp":
+        base = torch.zeros_like(base)
+    cur = base + synth.sweep_delta(dist, n, DEV, synth.SEED0 + 5 + logn)
+    bh, ch = to_np(base), to_np(cur)
+    got, _ = gpu_compress(lc, base, cur, nbits)
+    want = oracle.compress(bh, ch, nbits, threads=ORACLE_THREADS)
+    assert got.size == want.size and got.tobytes() == want.tobytes()
+    s = torch.from_numpy(got).to(DEV)
+    for k in (1, 3):
+        out = to_np(lc.recover(base, [s] * k))
+        ref = oracle.recover(bh, [want] * k, threads=ORACLE_THREADS)
+        assert np.array_equal(out.view(np.uint32), ref.view(np.uint32))
 
 
 def test_large_deltas_bypass_the_key_plane(lc, oracle):
@@ -271,8 +297,9 @@ def test_config_vgg16(lc, oracle):
 def test_config_xfmr1p3b_full_size(lc, oracle):
     """The benchmark's workload at full size: 1,315,575,808 elements, nbits 5, chain of 4.
 
-    Tables and statistics are compared in full; the payload on sampled chunks (the oracle codes only
-    those); the recovered state in full against Algorithm 1 step 7 computed directly on the CPU.
+    Every stream of the chain is compared byte for byte with the oracle's (coded with all host cores), after
+    the statistics and the table, so that a failure names the step; sampled chunks are also coded one by one;
+    the recovered state is compared in full against Algorithm 1 step 7 computed directly on the CPU.
     """
     from paper_2009_13003_b200 import synth
 
@@ -327,6 +354,14 @@ def test_config_xfmr1p3b_full_size(lc, oracle):
             assert np.array_equal(lane_bits[c], olane[k]), c
             lo = info.payload_offset + int(chunk_off[c])
             assert to_np(s[lo: lo + opay[k].size]).tobytes() == opay[k].tobytes(), c
+        # the whole stream
+        want = oracle.compress(tracked_h, u_h, nbits, threads=ORACLE_THREADS)
+        assert want.size == info.total_bytes
+        got = to_np(s)
+        step = 1 << 28
+        for lo in range(0, want.size, step):
+            assert got[lo: lo + step].tobytes() == want[lo: lo + step].tobytes(), "stream %d differs near byte %d" % (t, lo)
+        del want, got
         # tracked state: GPU recover vs step 7 computed directly
         tracked_h = oracle.apply_quantized(tracked_h, u_h, nbits)
         lc.recover(tracked, [s], out=tracked, workspace=ws)
