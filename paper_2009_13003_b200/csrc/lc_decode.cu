@@ -408,12 +408,15 @@ __device__ __noinline__ void decode_chunk_global(const StreamState* S, GlobalChu
 template <int KS>
 __global__ void __launch_bounds__(kDecMaxThreads, 1)
 decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, int32_t* __restrict__ status,
-              uint32_t stage_bytes) {
+              const uint32_t* __restrict__ flags, uint32_t stage_bytes) {
   // dynamic shared memory: [pad to 8 KB | 2 tables per stream | StreamState per stream | staging areas]
   extern __shared__ __align__(16) unsigned char s_raw[];
   unsigned char* tables = s_raw + ((kTableBytes - (smem_addr(s_raw) & (kTableBytes - 1))) & (kTableBytes - 1));
   StreamState* S = reinterpret_cast<StreamState*>(s_raw + kTableBytes + KS * 2 * kTableBytes);
   __shared__ int s_err;
+  // the prepare kernel has looked at the streams: this kernel runs only if one of them has more than 32 symbols
+  // (otherwise the pair decoder does the work) and none was rejected; the same word for every thread
+  if (*flags != kDecodeFlagGeneral) return;
 
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
@@ -501,7 +504,7 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
 
 template <int KS>
 cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, uint64_t n, float* out,
-                             int32_t* status, cudaStream_t cs) {
+                             int32_t* status, const uint32_t* flags, cudaStream_t cs) {
   static int sms_of[kMaxDevices] = {};  // by device ordinal; non-zero once the kernel's attributes are set there
   constexpr uint32_t kTables = kTableBytes + KS * (2 * kTableBytes + sizeof(StreamState));
   constexpr uint32_t kMaxDyn = kSmemPerSm - 1024 - kOverrunBytes;  // room for static __shared__ and the padding
@@ -579,19 +582,19 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
     if (cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributePreferredSharedMemoryCarveout, carve) != cudaSuccess)
       return cudaErrorUnknown;
   }
-  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, stage);
+  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, flags, stage);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
-                          int32_t* status, cudaStream_t cs) {
+                          int32_t* status, const uint32_t* flags, cudaStream_t cs) {
   switch (k) {
-    case 1: return launch_decode_ks<1>(base, streams, n, out, status, cs);
-    case 2: return launch_decode_ks<2>(base, streams, n, out, status, cs);
-    case 3: return launch_decode_ks<3>(base, streams, n, out, status, cs);
-    case 4: return launch_decode_ks<4>(base, streams, n, out, status, cs);
+    case 1: return launch_decode_ks<1>(base, streams, n, out, status, flags, cs);
+    case 2: return launch_decode_ks<2>(base, streams, n, out, status, flags, cs);
+    case 3: return launch_decode_ks<3>(base, streams, n, out, status, flags, cs);
+    case 4: return launch_decode_ks<4>(base, streams, n, out, status, flags, cs);
     default: return cudaErrorInvalidValue;
   }
 }
