@@ -18,7 +18,7 @@ constexpr uint32_t kTableEntryBytes = 16;
 constexpr uint32_t kPayloadAlign = 16;
 constexpr uint32_t kKeys = 512;  // 256*sign + exponent field
 
-__host__ __device__ constexpr inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+__host__ __device__ inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 struct StreamLayout {
   uint64_t nchunks, table_off, chunk_index_off, lane_index_off, payload_off;
@@ -71,7 +71,7 @@ struct Control {
   uint32_t max_len;       // written by the table kernel
   uint64_t payload_bits;  // written by the table kernel
   uint32_t wide;          // written by the table kernel: some delta has an exponent field >= 128
-  uint32_t decode_flags;  // lc_recover: written by the prepare kernel, tells the two decode kernels which one runs
+  uint32_t pad32_;
   uint64_t pad_[28];
   unsigned long long count[kKeys];  // elements per key
   uint32_t inv_min[kKeys];          // max over the bucket of ~bits (zero-initialised running minimum)
@@ -80,24 +80,17 @@ struct Control {
 };
 static_assert(sizeof(Control) % 256 == 0, "control block must keep the planes 256-byte aligned");
 
-// lc_recover keeps the decode tables of the (at most four) streams of one launch behind the control block, at an
-// offset that does not depend on n. decode_flags: 0 = the pair decoder runs (every stream valid, at most 32 symbols).
-constexpr uint32_t kDecodeTableBytes = 72 * 1024;
-constexpr uint32_t kDecodeFlagError = 1;    // a stream was rejected: neither decode kernel runs
-constexpr uint32_t kDecodeFlagGeneral = 2;  // some stream has more than 32 symbols: the general decoder runs
-
 struct WorkspaceLayout {
-  uint64_t control_off, decode_off, tiles_off, plane_off, total;
+  uint64_t control_off, tiles_off, plane_off, total;
   uint64_t nchunks, nunits;
 };
 
-__host__ __device__ constexpr inline WorkspaceLayout workspace_layout(uint64_t n) {
-  WorkspaceLayout W{};
+__host__ __device__ inline WorkspaceLayout workspace_layout(uint64_t n) {
+  WorkspaceLayout W;
   W.nchunks = (n + kChunkElems - 1) / kChunkElems;
   W.nunits = W.nchunks * kUnitsPerChunk;
   W.control_off = 0;
-  W.decode_off = sizeof(Control);
-  W.tiles_off = W.decode_off + kDecodeTableBytes;               // one 8-byte descriptor per chunk
+  W.tiles_off = sizeof(Control);                                // one 8-byte descriptor per chunk
   W.plane_off = align_up(W.tiles_off + 8 * W.nchunks, 256);
   W.total = align_up(W.plane_off + W.nchunks * kChunkElems, 256);  // 1 byte per element, whole chunks
   return W;
@@ -137,14 +130,7 @@ struct DecodeStreams {
   const uint8_t* ptr[4];
   uint64_t bytes[4];
 };
-// The recovery pass of up to four streams is three launches: the prepare kernel validates the streams, builds the
-// pair decoder's tables in `tables` (kDecodeTableBytes of the workspace) and sets *flags; then the pair decoder and
-// the general decoder, of which the one that *flags does not name returns at once.
-cudaError_t launch_decode_prepare(const DecodeStreams& streams, int k, uint64_t n, void* tables, uint32_t* flags,
-                                  int32_t* status, cudaStream_t cs);
-cudaError_t launch_decode_pairs(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
-                                int32_t* status, const void* tables, const uint32_t* flags, cudaStream_t cs);
 cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
-                          int32_t* status, const uint32_t* flags, cudaStream_t cs);
+                          int32_t* status, cudaStream_t cs);
 
 }  // namespace lc

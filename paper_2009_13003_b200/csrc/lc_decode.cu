@@ -39,11 +39,19 @@ using namespace dec;
 constexpr int kDecMaxThreads = 512;
 constexpr int kL1Bits = 6;
 constexpr int kL1Rep = 16;
-constexpr int kSubBitsMax = 6;                     // second level: the next 6 bits (5 or 4 if many prefixes need one)
+// Second level: one sub-table per 6-bit prefix that belongs to longer codes, all of one depth: the next 10 bits if a
+// single prefix needs one (8 KB hold one table of 1024 entries; a Huffman code's long codes usually hang under one
+// prefix), down to the next 4 bits if every prefix does (64 tables of 16 entries).
+constexpr int kSubBitsMax = 10;
 constexpr int kSubBitsMin = 4;
 constexpr int kL2Bits = kL1Bits + kSubBitsMax;     // longest code the two table levels resolve
-constexpr uint32_t kLongCode = 0xFFFFFFFFu;
-static_assert(2 * kL2Bits <= 33, "two table-resolved codes must fit the refill guarantee");
+static_assert(kL2Bits <= 16, "the second code of a pair is looked up in the 32-bit upper word behind the first");
+static_assert(((1 << kL1Bits) << (kSubBitsMin + 3)) <= 8192, "at the smallest depth every prefix gets a sub-table");
+// Length field of a table entry that does not resolve its code. As a length it takes the bit count far below zero,
+// which is how the hot loop notices: a step subtracts at most four of them per stream, and 1..4 times 2^29 (less a
+// few real lengths) leaves the sign bit of the 32-bit count set in every case.
+constexpr uint32_t kLongCode = 0x20000000u;
+constexpr int kPrefetchRows = 8;  // distance, in steps of 512 bytes per warp, of the L2 prefetch of base
 
 // The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory.
 constexpr uint32_t kTableBytes = 8192;
@@ -64,7 +72,7 @@ struct alignas(16) StreamState {
   // validation accumulators
   unsigned long long kraft, count_sum, bit_sum;
   uint32_t seen_max, nused, nsub;
-  uint32_t sub_bits;  // 6, 5 or 4: 16, 32 or 64 sub-tables, the last of which only says "longer"
+  uint32_t sub_bits;  // depth of the sub-tables, kSubBitsMin..kSubBitsMax: as many as 8 KB hold at that depth
   uint8_t sub_of_prefix[1 << kL1Bits], prefix_of_sub[1 << kL1Bits];
   uint8_t sym_len[256];   // code length by symbol id
   uint32_t miss_count[2];  // first-level prefixes without a short code, per warp of 32 prefixes
@@ -200,7 +208,7 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
 
   // ---- lookup tables: canonical decode of each entry's own index
   // First-level prefixes that belong to longer codes get a sub-table each. Sub-tables are as deep as
-  // their number allows (8 KB in all, one kept as the table that only says "longer").
+  // their number allows (8 KB in all).
   {
     const bool miss = tid < (1 << kL1Bits) && S.nused >= 2 && canonical_lookup(S, tid, kL1Bits).y == 0;
     const uint32_t ballot = __ballot_sync(0xffffffffu, miss);
@@ -209,10 +217,10 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
     if (tid < (1 << kL1Bits)) {
       const uint32_t misses = S.miss_count[0] + S.miss_count[1];
       uint32_t sub_bits = kSubBitsMax;
-      while (sub_bits > kSubBitsMin && misses > (kTableBytes >> (sub_bits + 3)) - 1) sub_bits -= 1;
-      const uint32_t usable = (kTableBytes >> (sub_bits + 3)) - 1;
+      while (sub_bits > kSubBitsMin && misses > (kTableBytes >> (sub_bits + 3))) sub_bits -= 1;
+      const uint32_t usable = kTableBytes >> (sub_bits + 3);  // >= misses: every such prefix gets a table
       const uint32_t rank = __popc(ballot & ((1u << (tid & 31)) - 1)) + (tid >= 32 ? S.miss_count[0] : 0u);
-      uint32_t sub = usable;  // the "longer" sub-table
+      uint32_t sub = 0;
       if (miss && rank < usable) {
         sub = rank;
         S.prefix_of_sub[sub] = (uint8_t)tid;
@@ -322,12 +330,23 @@ __device__ __forceinline__ uint32_t long_code(LaneBits<STAGED>& B, const StreamS
   return rep;
 }
 
-// Full chunk: the hot loop. Per step a lane decodes 4 elements x KS streams; the KS streams are
-// independent dependency chains and are written interleaved.
+// Full chunk: the hot loop. Per step a lane decodes 4 elements x KS streams; the KS streams are independent
+// dependency chains and are written interleaved.
+//
+// The loop body is straight-line code. A lane tops its bit buffers up once per step and then decodes its four
+// codes per stream from the upper word alone, two at a time (the second lookup takes the first code's length,
+// the buffer is shifted once per pair). Two things can go wrong for a lane in a step, both rare: a code longer
+// than the tables resolve, and four codes that take more bits than the buffer held (32 are guaranteed, four
+// table-resolved codes can take 64). Both show as a negative bit count at the end of the step: the marker of an
+// unresolved code is a huge length, and a lookup on too few valid bits always overdraws, because no code is a
+// prefix of another. One warp vote per step finds them, and the flagged lanes decode the step again from where it
+// started, one code at a time with a top-up before each (a top-up makes 32 bits valid, a table-resolved code
+// takes at most 16). Whatever the quick pass did to their buffers in
+// between stays inside the staged chunk (a top-up moves one word per step) and is discarded.
 template <int KS, bool STAGED>
 __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const Source* W, const uint32_t* start,
                                                     const float* base, float* out, uint64_t c, uint32_t lane,
-                                                    int32_t* status) {
+                                                    const float* next_rows, int32_t* status) {
   LaneBits<STAGED> bits[KS];
   // the streams' tables follow each other at 2 * kTableBytes: one base address, the rest as immediate offsets
   const uint32_t l1lane = smem_addr(S[0].l1) | ((lane & (kL1Rep - 1)) * 8u);
@@ -339,36 +358,83 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
   }
   const uint64_t e0 = c * kChunkElems + 4 * lane;
   float4 b = ldg_stream_v4(base + e0);
+  // Rows of base are asked into the L2 kPrefetchRows steps before they are loaded: a warp has one row in
+  // registers ahead of its use, which alone leaves far too few bytes in flight per SM for the DRAM latency.
+  // Behind this chunk's last row the requests go on with the first rows of the chunk this warp decodes next
+  // (`next_rows`: this lane's part of that chunk's first row, or of this chunk's first row if there is none).
+  const float* pf = base + e0 + 128 * kPrefetchRows;
 #pragma unroll 1
   for (uint32_t j = 0; j < kSteps; ++j) {
     const uint64_t i = e0 + 128ull * j;
     float x[4] = {b.x, b.y, b.z, b.w};
     // next step's 16 bytes of base, requested a whole step ahead (the last step re-reads its own)
     b = ldg_stream_v4(base + i + (j + 1 < kSteps ? 128 : 0));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(pf));
+    pf = (j == kSteps - kPrefetchRows - 1) ? next_rows : pf + 128;
+    int cnt0[KS];
+    uint32_t next0[KS];
+    uint32_t flags = 0;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      if ((e & 1) == 0) {
+    for (int s = 0; s < KS; ++s) {
+      cnt0[s] = bits[s].cnt;  // where the step starts, for the careful pass
+      next0[s] = bits[s].next;
+      bits[s].refill(W[s]);
+    }
 #pragma unroll
-        for (int s = 0; s < KS; ++s) bits[s].refill(W[s]);
-      }
-      uint2 ent[KS];
-      uint32_t longest = 0;
-      ent[0] = lookup_code<0>(bits[0].hi, l1lane, sub_shift[0]);
-      if (KS > 1) ent[1 % KS] = lookup_code<2 * kTableBytes>(bits[1 % KS].hi, l1lane, sub_shift[1 % KS]);
-      if (KS > 2) ent[2 % KS] = lookup_code<4 * kTableBytes>(bits[2 % KS].hi, l1lane, sub_shift[2 % KS]);
-      if (KS > 3) ent[3 % KS] = lookup_code<6 * kTableBytes>(bits[3 % KS].hi, l1lane, sub_shift[3 % KS]);
+    for (int h = 0; h < 2; ++h) {
+      uint2 ea[KS], eb[KS];
+      uint32_t h1[KS];
+      ea[0] = lookup_code<0>(bits[0].hi, l1lane, sub_shift[0]);
+      if (KS > 1) ea[1 % KS] = lookup_code<2 * kTableBytes>(bits[1 % KS].hi, l1lane, sub_shift[1 % KS]);
+      if (KS > 2) ea[2 % KS] = lookup_code<4 * kTableBytes>(bits[2 % KS].hi, l1lane, sub_shift[2 % KS]);
+      if (KS > 3) ea[3 % KS] = lookup_code<6 * kTableBytes>(bits[3 % KS].hi, l1lane, sub_shift[3 % KS]);
 #pragma unroll
-      for (int s = 0; s < KS; ++s) longest |= ent[s].y;  // lengths are < 64, the marker is all ones
-      if (__builtin_expect(__any_sync(0xffffffffu, longest > 63u), 0)) {
-#pragma unroll
-        for (int s = 0; s < KS; ++s) {
-          if (ent[s].y > 63u) ent[s] = make_uint2(long_code<STAGED>(bits[s], S[s], W[s], status), 0u);  // consumed
-        }
-      }
+      for (int s = 0; s < KS; ++s) h1[s] = __funnelshift_l(0u, bits[s].hi, ea[s].y);  // hi << length (mod 32)
+      eb[0] = lookup_code<0>(h1[0], l1lane, sub_shift[0]);
+      if (KS > 1) eb[1 % KS] = lookup_code<2 * kTableBytes>(h1[1 % KS], l1lane, sub_shift[1 % KS]);
+      if (KS > 2) eb[2 % KS] = lookup_code<4 * kTableBytes>(h1[2 % KS], l1lane, sub_shift[2 % KS]);
+      if (KS > 3) eb[3 % KS] = lookup_code<6 * kTableBytes>(h1[3 % KS], l1lane, sub_shift[3 % KS]);
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        x[e] = __fadd_rn(x[e], __uint_as_float(ent[s].x));
-        bits[s].consume(ent[s].y);
+        x[2 * h] = __fadd_rn(x[2 * h], __uint_as_float(ea[s].x));
+        x[2 * h + 1] = __fadd_rn(x[2 * h + 1], __uint_as_float(eb[s].x));
+        const uint32_t len = ea[s].y + eb[s].y;
+        bits[s].hi = __funnelshift_l(bits[s].lo, bits[s].hi, len);
+        bits[s].lo = __funnelshift_l(0u, bits[s].lo, len);
+        bits[s].cnt = (int)((uint32_t)bits[s].cnt - len);
+      }
+    }
+#pragma unroll
+    for (int s = 0; s < KS; ++s) flags |= (uint32_t)bits[s].cnt;
+    if (__builtin_expect(__any_sync(0xffffffffu, (int)flags < 0), 0)) {
+      if ((int)flags < 0) {
+        const float4 b0 = ldg_stream_v4(base + i);
+        x[0] = b0.x; x[1] = b0.y; x[2] = b0.z; x[3] = b0.w;
+#pragma unroll
+        for (int s = 0; s < KS; ++s) {
+          bits[s].cnt = cnt0[s];
+          bits[s].next = next0[s];
+          bits[s].seek(W[s], bits[s].bitpos(W[s]));
+        }
+        // one element per trip; x is rotated so that the loop needs no indexed register
+#pragma unroll 1
+        for (int e = 0; e < 4; ++e) {
+          float v = x[0];
+          uint2 ent[KS];
+#pragma unroll
+          for (int s = 0; s < KS; ++s) bits[s].refill(W[s]);
+          ent[0] = lookup_code<0>(bits[0].hi, l1lane, sub_shift[0]);
+          if (KS > 1) ent[1 % KS] = lookup_code<2 * kTableBytes>(bits[1 % KS].hi, l1lane, sub_shift[1 % KS]);
+          if (KS > 2) ent[2 % KS] = lookup_code<4 * kTableBytes>(bits[2 % KS].hi, l1lane, sub_shift[2 % KS]);
+          if (KS > 3) ent[3 % KS] = lookup_code<6 * kTableBytes>(bits[3 % KS].hi, l1lane, sub_shift[3 % KS]);
+#pragma unroll
+          for (int s = 0; s < KS; ++s) {
+            if (ent[s].y > 63u) ent[s] = make_uint2(long_code<STAGED>(bits[s], S[s], W[s], status), 0u);  // consumed
+            v = __fadd_rn(v, __uint_as_float(ent[s].x));
+            bits[s].consume(ent[s].y);
+          }
+          x[0] = x[1]; x[1] = x[2]; x[2] = x[3]; x[3] = v;
+        }
       }
     }
     *reinterpret_cast<float4*>(out + i) = make_float4(x[0], x[1], x[2], x[3]);
@@ -408,15 +474,12 @@ __device__ __noinline__ void decode_chunk_global(const StreamState* S, GlobalChu
 template <int KS>
 __global__ void __launch_bounds__(kDecMaxThreads, 1)
 decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, int32_t* __restrict__ status,
-              const uint32_t* __restrict__ flags, uint32_t stage_bytes) {
+              uint32_t stage_bytes) {
   // dynamic shared memory: [pad to 8 KB | 2 tables per stream | StreamState per stream | staging areas]
   extern __shared__ __align__(16) unsigned char s_raw[];
   unsigned char* tables = s_raw + ((kTableBytes - (smem_addr(s_raw) & (kTableBytes - 1))) & (kTableBytes - 1));
   StreamState* S = reinterpret_cast<StreamState*>(s_raw + kTableBytes + KS * 2 * kTableBytes);
   __shared__ int s_err;
-  // the prepare kernel has looked at the streams: this kernel runs only if one of them has more than 32 symbols
-  // (otherwise the pair decoder does the work) and none was rejected; the same word for every thread
-  if (*flags != kDecodeFlagGeneral) return;
 
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
@@ -487,8 +550,11 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
     cp_async_wait_all();
     __syncwarp();
     if ((c + 1) * kChunkElems <= n) {
-      if (fits) decode_chunk_fast<KS, true>(S, W, start, base, out, c, lane, status);
-      else decode_chunk_fast<KS, false>(S, W, start, base, out, c, lane, status);
+      // where the L2 prefetch goes on behind this chunk: the next chunk of this warp, if it is a full one
+      const uint64_t cn = c + nwarps;
+      const float* next_rows = base + ((cn + 1) * kChunkElems <= n ? cn : c) * kChunkElems + 4 * lane;
+      if (fits) decode_chunk_fast<KS, true>(S, W, start, base, out, c, lane, next_rows, status);
+      else decode_chunk_fast<KS, false>(S, W, start, base, out, c, lane, next_rows, status);
     } else {
       GlobalChunk G;
 #pragma unroll
@@ -504,7 +570,7 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
 
 template <int KS>
 cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, uint64_t n, float* out,
-                             int32_t* status, const uint32_t* flags, cudaStream_t cs) {
+                             int32_t* status, cudaStream_t cs) {
   static int sms_of[kMaxDevices] = {};  // by device ordinal; non-zero once the kernel's attributes are set there
   constexpr uint32_t kTables = kTableBytes + KS * (2 * kTableBytes + sizeof(StreamState));
   constexpr uint32_t kMaxDyn = kSmemPerSm - 1024 - kOverrunBytes;  // room for static __shared__ and the padding
@@ -582,19 +648,19 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
     if (cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributePreferredSharedMemoryCarveout, carve) != cudaSuccess)
       return cudaErrorUnknown;
   }
-  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, flags, stage);
+  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, stage);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
-                          int32_t* status, const uint32_t* flags, cudaStream_t cs) {
+                          int32_t* status, cudaStream_t cs) {
   switch (k) {
-    case 1: return launch_decode_ks<1>(base, streams, n, out, status, flags, cs);
-    case 2: return launch_decode_ks<2>(base, streams, n, out, status, flags, cs);
-    case 3: return launch_decode_ks<3>(base, streams, n, out, status, flags, cs);
-    case 4: return launch_decode_ks<4>(base, streams, n, out, status, flags, cs);
+    case 1: return launch_decode_ks<1>(base, streams, n, out, status, cs);
+    case 2: return launch_decode_ks<2>(base, streams, n, out, status, cs);
+    case 3: return launch_decode_ks<3>(base, streams, n, out, status, cs);
+    case 4: return launch_decode_ks<4>(base, streams, n, out, status, cs);
     default: return cudaErrorInvalidValue;
   }
 }
