@@ -37,16 +37,28 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def source_digest(cu_file):
+    import hashlib
+
+    path = os.path.join(ROOT, "paper_2009_13003_b200", "csrc", cu_file)
+    with open(path, "rb") as f:
+        return hashlib.sha1(f.read()).hexdigest()[:12]
+
+
 def measured_traffic(kernel, n):
-    """DRAM bytes per launch of `kernel` from the committed ncu capture (profiles/traffic.txt holds bytes per
-    element measured on a smaller case; every pass is a linear scan, so traffic scales with n). None if absent."""
+    """DRAM bytes per launch of `kernel` from the committed ncu capture. profiles/traffic.txt holds, per kernel,
+    bytes per element measured on a smaller case (every pass is a linear scan, so traffic scales with n), the
+    source file of the kernel and that file's digest when the counters were taken. None if there is no entry or
+    the kernel's source has changed since."""
     try:
         with open(os.path.join(ROOT, "profiles", "traffic.txt")) as f:
-            table = dict(line.split() for line in f if line.strip() and not line.startswith("#"))
-        per_elem = table.get(kernel.split("<")[0])
-        return None if per_elem is None else float(per_elem) * n
+            for line in f:
+                parts = line.split()
+                if len(parts) == 4 and not line.startswith("#") and parts[0] == kernel.split("<")[0]:
+                    return float(parts[1]) * n if source_digest(parts[2]) == parts[3] else None
     except Exception:
-        return None
+        pass
+    return None
 
 
 # ------------------------------------------------------------------------------------------- clocks
@@ -63,15 +75,18 @@ class ClockSampler:
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index):
+    def __init__(self, gpu_id):
+        """gpu_id: what `nvidia-smi -i` takes. Pass the device's UUID: with CUDA_VISIBLE_DEVICES set, a CUDA ordinal
+        is not nvidia-smi's index, and the samples would be another GPU's."""
         import threading
 
         self.lines = []  # (arrival time, text)
         self.t_start = None
         self.proc = None
+        self.gpu_id = str(gpu_id)
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                ["nvidia-smi", "-i", self.gpu_id, "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
                  "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -92,7 +107,7 @@ class ClockSampler:
 
     def stop(self):
         t_end = time.perf_counter()
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "gpu": self.gpu_id}
         if self.proc is None:
             return out
         time.sleep(0.03)
@@ -121,6 +136,16 @@ class ClockSampler:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
         out["reasons"] = sorted(reasons)
         return out
+
+
+def gpu_uuid(cuda_ordinal):
+    """'GPU-<uuid>' of a CUDA device, the form nvidia-smi -i accepts; the ordinal itself if torch cannot tell."""
+    try:
+        import torch
+
+        return "GPU-" + str(torch.cuda.get_device_properties(cuda_ordinal).uuid)
+    except Exception:
+        return str(cuda_ordinal)
 
 
 # ------------------------------------------------------------------------------------------- N > 1
@@ -168,69 +193,101 @@ def aggregate_value(units_per_rank, world, max_ms):
 # ------------------------------------------------------------------------------------------- arms
 
 
-def run_reference(args, rank):
-    """The CPU oracle, as it stands, timed on a bounded sample of the workload (rank 0 only)."""
-    if rank != 0:
-        return None
-    import numpy as np  # noqa: F401
+def host_threads():
+    """Threads the oracle's chunk-parallel mode gets: the cores this process may run on."""
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except Exception:
+        return max(1, os.cpu_count() or 1)
 
+
+ONE_CORE_SAMPLE_ELEMS = 1 << 25  # the single-threaded figure is taken on the first 33,554,432 elements
+
+
+def oracle_sample_chain(cfg, m, threads):
+    """Host copy of the workload's first m elements, tracked through cfg.chain snapshots the way Algorithm 1 does,
+    by the oracle. Returns (u0, tracked state before the last snapshot, last state, streams). The sample is coded on
+    its own: a stream's table depends on the whole vector it codes."""
     from oracle import lc_oracle
     from paper_2009_13003_b200 import synth
 
-    cfg = synth.CONFIGS[WORKLOAD]
-    # bounded sample: the oracle does about 12 M elements per second of (compress + chain-of-4 recover) on one
-    # core, and the whole run (set-up, warm-up, steps) should end within a few minutes
-    budget_s = 150.0
-    m = int(budget_s / (args.steps + args.warmup + 2) * 12e6) // 4096 * 4096
-    m = max(4096, min(CPU_SAMPLE_ELEMS, m, cfg.n))
     u0 = synth.base_state(cfg, "cpu", m).numpy()
     tracked, u, streams = u0.copy(), u0.copy(), []
     for t in range(1, cfg.chain + 1):
         u = u + synth.snapshot_delta(cfg, t, "cpu", m).numpy()
-        s = lc_oracle.compress(tracked, u, cfg.nbits)
+        s = lc_oracle.compress(tracked, u, cfg.nbits, threads=threads)
         streams.append(s)
         if t < cfg.chain:
-            tracked = lc_oracle.recover(tracked, [s])
+            tracked = lc_oracle.recover(tracked, [s], threads=threads)
+    return u0, tracked, u, streams
+
+
+def time_oracle(cfg, u0, tracked, u, streams, threads, repeats=1):
+    """Seconds of one oracle compress of the last snapshot and of one recovery of the whole chain (best of repeats)."""
+    from oracle import lc_oracle
+
+    t_c = t_r = float("inf")
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        lc_oracle.compress(tracked, u, cfg.nbits, threads=threads)
+        t1 = time.perf_counter()
+        lc_oracle.recover(u0, streams, threads=threads)
+        t2 = time.perf_counter()
+        t_c, t_r = min(t_c, t1 - t0), min(t_r, t2 - t1)
+    return t_c, t_r
+
+
+def oracle_baseline(cfg, n):
+    """The cpu_baseline object: the oracle, as it stands, on the first CPU_SAMPLE_ELEMS elements of the workload with
+    all host cores (its chunk-parallel mode), and on a smaller sample with one core (its plain single-threaded pass).
+    Same sample and same mode as the `--impl reference` arm."""
+    m = min(CPU_SAMPLE_ELEMS, n)
+    threads = host_threads()
+    chain = oracle_sample_chain(cfg, m, threads)
+    t_c, t_r = time_oracle(cfg, *chain, threads=threads)
+    m1 = min(ONE_CORE_SAMPLE_ELEMS, n)
+    chain1 = oracle_sample_chain(cfg, m1, threads)
+    c1, r1 = time_oracle(cfg, *chain1, threads=None)
+    return {"value": 2 * 4 * m / (t_c + t_r) / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+            "sample": "first %d of %d elements: 1 compress (%.2f s) + 1 recover of a chain of %d (%.2f s), oracle's "
+                      "chunk-parallel mode on %d threads" % (m, n, t_c, cfg.chain, t_r, threads),
+            "compress_gbs": 4 * m / t_c / 1e9, "recover_gbs": 4 * m / t_r / 1e9,
+            "one_core": {"value": 2 * 4 * m1 / (c1 + r1) / 1e9, "unit": "GB/s", "cores": 1,
+                         "sample": "first %d elements, plain single-threaded oracle: compress %.2f s, recover %.2f s"
+                                   % (m1, c1, r1),
+                         "compress_gbs": 4 * m1 / c1 / 1e9, "recover_gbs": 4 * m1 / r1 / 1e9}}
+
+
+def run_reference(args, rank):
+    """The CPU oracle, as it stands, timed on a bounded sample of the workload (rank 0 only): every step is one
+    compress + one recovery of the chain on the first CPU_SAMPLE_ELEMS elements, with all host cores."""
+    if rank != 0:
+        return None
+    from paper_2009_13003_b200 import synth
+
+    cfg = synth.CONFIGS[WORKLOAD]
+    m = min(CPU_SAMPLE_ELEMS, cfg.n)
+    threads = host_threads()
+    chain = oracle_sample_chain(cfg, m, threads)
     times = []
     for it in range(args.warmup + args.steps):
-        t0 = time.perf_counter()
-        lc_oracle.compress(tracked, u, cfg.nbits)
-        lc_oracle.recover(u0, streams)
+        t_c, t_r = time_oracle(cfg, *chain, threads=threads)
         if it >= args.warmup:
-            times.append(time.perf_counter() - t0)
+            times.append(t_c + t_r)
     ms = 1e3 * sum(times) / len(times)
     value = 2 * 4 * m / (ms * 1e-3) / 1e9
-    sample = "first %d of %d elements, compress + recover(chain 4) per step" % (m, cfg.n)
+    sample = ("first %d of %d elements, compress + recover(chain %d) per step, oracle's chunk-parallel mode on %d "
+              "threads" % (m, cfg.n, cfg.chain, threads))
     return {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "n": cfg.n, "nbits": cfg.nbits, "recover_chain": cfg.chain,
                    "sample_elems": m},
-        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
-
-
-def time_oracle_sample(cfg, n, u0, tracked, u, streams_dev):
-    """cpu_baseline leg: the oracle on the first CPU_SAMPLE_ELEMS elements of the same device inputs."""
-    from oracle import lc_oracle
-
-    m = min(CPU_SAMPLE_ELEMS, n)
-    u0_h, tr_h, u_h = (x[:m].cpu().numpy() for x in (u0, tracked, u))
-    # the sample's own chain (tables depend on the whole vector, so the sample is coded on its own)
-    t0 = time.perf_counter()
-    s = lc_oracle.compress(tr_h, u_h, cfg.nbits)
-    t_c = time.perf_counter() - t0
-    t0 = time.perf_counter()
-    lc_oracle.recover(u0_h, [s] * cfg.chain)
-    t_r = time.perf_counter() - t0
-    value = 2 * 4 * m / (t_c + t_r) / 1e9
-    return {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle",
-            "sample": "first %d of %d elements: 1 compress (%.2f s) + 1 recover of a chain of %d (%.2f s)"
-                      % (m, n, t_c, cfg.chain, t_r),
-            "compress_gbs": 4 * m / t_c / 1e9, "recover_gbs": 4 * m / t_r / 1e9}
 
 
 def run_ours(args, rank, world, local_rank):
@@ -285,7 +342,7 @@ def run_ours(args, rank, world, local_rank):
         lc.compress_async(tracked, u, nbits, sbuf, ws)
         recover_chain(out)
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    sampler = ClockSampler(gpu_uuid(local_rank)) if rank == 0 else None
     for _ in range(args.warmup):
         step()
     torch.cuda.synchronize()
@@ -347,6 +404,23 @@ def run_ours(args, rank, world, local_rank):
     assert lc.last_status(ws) == 0
     assert torch.equal(sbuf[: stream_bytes[-1]], streams[-1]), "fused compress did not reproduce the stream"
     recover_chain(out)  # `out` holds the whole chain's result again
+    # ---- checkpoint merging (Section 3.2): the chain as one super-step stream; outside the timed region
+    merge_ms = merged_bytes = None
+    if chain <= lc.MAX_CHAIN:
+        mg = []
+        scratch = torch.empty_like(u0)
+        for _ in range(4):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            lc.merge_async(u0, streams, nbits, sbuf, scratch, ws)
+            b.record()
+            torch.cuda.synchronize()
+            mg.append(a.elapsed_time(b))
+        assert lc.last_status(ws) == 0
+        merge_ms = statistics.median(mg[1:])
+        merged_bytes = int(lc.stream_info(sbuf).total_bytes)
+        assert torch.equal(scratch, out), "merge did not recover the chain's state"
+        del scratch
 
     # ---- end to end through the host-buffer entry points (pinned host memory, copies inside)
     e2e = None
@@ -378,6 +452,15 @@ def run_ours(args, rank, world, local_rank):
         return None
 
     peak, peak_kind = measured_peak()
+    nominal = 8000.0  # GB/s, the HBM3e figure the target is worded against; fractions of it beside the measured ones
+    # entropy of the last stream's symbols, from the counts in its symbol table (what a Huffman code can approach)
+    import numpy as np
+
+    tab = np.frombuffer(streams[-1][64: 64 + 16 * nsym].cpu().numpy().tobytes(),
+                        dtype=[("key", "<u2"), ("len", "u1"), ("pad", "u1"), ("rep", "<u4"), ("count", "<u8")])
+    pr = tab["count"][tab["count"] > 0].astype(np.float64) / n
+    entropy_bits = float(-(pr * np.log2(pr)).sum())
+    code_bits = float((tab["count"].astype(np.float64) * tab["len"]).sum() / n)
     decode_launches = sum((min(lc.MAX_CHAIN, chain - f) + 3) // 4 for f in range(0, chain, lc.MAX_CHAIN))
     sbar = [b / n for b in stream_bytes]
     kernels = {
@@ -389,6 +472,7 @@ def run_ours(args, rank, world, local_rank):
     achieved = kernels[dom]["alg_bytes"] / (kernels[dom]["ms"] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_kind + " (STREAM-style copy)",
+                "frac_of_nominal_8tbs": achieved / nominal,
                 "traffic": measured_traffic(dom, n),
                 "per_kernel": {k: {"ms": v["ms"], "achieved_gbs": v["alg_bytes"] / (v["ms"] * 1e-3) / 1e9,
                                    "frac": v["alg_bytes"] / (v["ms"] * 1e-3) / 1e9 / peak}
@@ -404,23 +488,29 @@ def run_ours(args, rank, world, local_rank):
                    else "vectors fit the 126 MB L2: L2-resident figures",
                    "replicas": world},
         "compress": {"ms": comp, "state_gbs": 4 * n / (comp * 1e-3) / 1e9, "alg_gbs": comp_alg,
-                     "frac_of_peak": comp_alg / peak,
+                     "frac_of_peak": comp_alg / peak, "frac_of_nominal_8tbs": comp_alg / nominal,
                      "kernels_ms": {"stats": stats_ms, "table": table_ms, "encode": encode_ms}},
         "recover": {"ms": rec, "state_gbs": 4 * n / (rec * 1e-3) / 1e9, "alg_gbs": rec_alg,
-                    "frac_of_peak": rec_alg / peak},
+                    "frac_of_peak": rec_alg / peak, "frac_of_nominal_8tbs": rec_alg / nominal},
         "recover_k1": {"ms": rec1_ms, "alg_gbs": (8.0 * n + stream_bytes[0]) / (rec1_ms * 1e-3) / 1e9,
                        "frac_of_peak": (8.0 * n + stream_bytes[0]) / (rec1_ms * 1e-3) / 1e9 / peak},
         # algorithmic bytes of the fused call: read base and cur, write the tracked state and the stream
         "compress_update": {"ms": cu_ms, "separate_calls_ms": comp + rec1_ms,
                             "alg_gbs": (12.0 * n + stream_bytes[-1]) / (cu_ms * 1e-3) / 1e9,
                             "frac_of_peak": (12.0 * n + stream_bytes[-1]) / (cu_ms * 1e-3) / 1e9 / peak},
-        "ratio": {"stream": 4.0 * n / stream_bytes[-1], "bits_per_element": 8.0 * sbar[-1]},
+        # algorithmic bytes of a merge: read base and the chain's streams, write the merged stream
+        "merge": None if merge_ms is None else {
+            "ms": merge_ms, "streams_in": chain, "merged_ratio": 4.0 * n / merged_bytes,
+            "alg_gbs": (4.0 * n + sum(stream_bytes) + merged_bytes) / (merge_ms * 1e-3) / 1e9,
+            "frac_of_peak": (4.0 * n + sum(stream_bytes) + merged_bytes) / (merge_ms * 1e-3) / 1e9 / peak},
+        "ratio": {"stream": 4.0 * n / stream_bytes[-1], "bits_per_element": 8.0 * sbar[-1],
+                  "code_bits_per_element": code_bits, "entropy_bits_per_element": entropy_bits},
         "size_model": size_model,
         "roofline": roofline, "clocks": clocks, "e2e": e2e,
-        "gpu_launches": (3 + decode_launches) * args.steps,  # stats, table, encode + decode launches per step
+        "gpu_launches": (3 + decode_launches) * args.steps,  # stats, table, encode + decode kernels per step
     }
     if world == 1 and not args.no_cpu_baseline:
-        result["cpu_baseline"] = time_oracle_sample(cfg, n, u0, tracked, u, streams)
+        result["cpu_baseline"] = oracle_baseline(cfg, n)
     return result
 
 
@@ -428,7 +518,8 @@ def run_sweep(args):
     """Sizes x distributions x nbits: compress and single-stream recover times and the ratio, as CSV on stdout.
 
     Not the benchmark line: a reference table (roofline curve over n and the degenerate cases). Vectors of
-    2^24 elements and fewer fit the 126 MB L2, so their figures are L2-resident.
+    2^24 elements and fewer fit the 126 MB L2, so their plain figures are L2-resident; for those sizes the table
+    also has cold figures, taken with the L2 flushed (a 256 MB buffer written) before every timed call.
     """
     import torch
 
@@ -439,7 +530,8 @@ def run_sweep(args):
     lc.lib()
     peak, _ = measured_peak()
     print("n,dist,nbits,compress_ms,recover_ms,compress_state_gbs,recover_state_gbs,compress_alg_frac,"
-          "recover_alg_frac,ratio,bits_per_element,nsym,max_len")
+          "recover_alg_frac,ratio,bits_per_element,nsym,max_len,compress_cold_ms,recover_cold_ms")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     for logn in (16, 20, 24, 28, 30):
         n = 1 << logn
         base = synth.normal(n, 0.02, dev, synth.SEED0 + 5)
@@ -476,10 +568,26 @@ def run_sweep(args):
                 assert lc.last_status(ws) == 0
                 c_ms, r_ms = statistics.median(times["c"]), statistics.median(times["r"])
                 sb = int(info.total_bytes)
-                print("%d,%s,%d,%.4f,%.4f,%.1f,%.1f,%.3f,%.3f,%.2f,%.3f,%d,%d" % (
+                cold = {"c": [], "r": []}
+                if logn <= 24:
+                    for it in range(5):
+                        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                        flush.zero_()
+                        e[0].record()
+                        lc.compress_async(b, cur, nbits, sbuf, ws)
+                        e[1].record()
+                        flush.zero_()
+                        e[2].record()
+                        lc.recover_async(b, [s], out, ws)
+                        e[3].record()
+                        torch.cuda.synchronize()
+                        cold["c"].append(e[0].elapsed_time(e[1]))
+                        cold["r"].append(e[2].elapsed_time(e[3]))
+                cc, cr = (("%.4f" % statistics.median(cold[k])) if cold[k] else "" for k in ("c", "r"))
+                print("%d,%s,%d,%.4f,%.4f,%.1f,%.1f,%.3f,%.3f,%.2f,%.3f,%d,%d,%s,%s" % (
                     n, dist, nbits, c_ms, r_ms, 4 * n / c_ms / 1e6, 4 * n / r_ms / 1e6,
                     (8.0 * n + sb) / c_ms / 1e6 / peak, (8.0 * n + sb) / r_ms / 1e6 / peak,
-                    4.0 * n / sb, 8.0 * sb / n, info.nsym, info.max_len), flush=True)
+                    4.0 * n / sb, 8.0 * sb / n, info.nsym, info.max_len, cc, cr), flush=True)
                 del sbuf
             del cur
         del base, ws, out

@@ -36,11 +36,13 @@ extern "C" {
 #define LC_ERR_MISMATCH (-5)  /* a stream's element count differs from n */
 #define LC_ERR_TIMEOUT (-6)   /* a bounded device-side wait gave up */
 #define LC_ERR_CUDA (-7)      /* a CUDA runtime call failed */
+#define LC_ERR_RANGE (-8)     /* lc_compress_async: some |delta| >= 2, which needs the live state after it was released */
 
 #define LC_MAX_CHAIN 8 /* most streams one lc_recover call applies */
 
-/* Same underlying type as cudaStream_t, so a cudaStream_t can be passed directly. */
+/* Same underlying types as cudaStream_t and cudaEvent_t, so those can be passed directly. */
 typedef struct CUstream_st* lc_cuda_stream_t;
+typedef struct CUevent_st* lc_cuda_event_t;
 
 /* Host copy of a stream header (format section 3.1). */
 typedef struct lc_info {
@@ -138,6 +140,46 @@ int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, 
  */
 int lc_recover(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k,
                uint64_t n, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs);
+
+/*
+ * Compress pass split over two CUDA streams (Section 3.2, "Asynchronous Execution": only the first step of the
+ * checkpointing process, the delta against the live model state, depends on that state; the rest can run beside
+ * the next training iteration).
+ * The statistics pass, the only one that reads base and cur, is enqueued on `cs_state` (the stream that owns the
+ * model state), followed by a record of `state_read` on that stream. The table and encode passes are enqueued on
+ * `cs_side` behind a wait for that event. Work enqueued on cs_state after this call therefore waits for the
+ * statistics pass only, and may overwrite cur (and base) as soon as it runs; the stream is complete when cs_side
+ * has drained.
+ *   state_read  an event created by the caller (cudaEventCreateWithFlags(..., cudaEventDisableTiming) is enough);
+ *               recorded by this call. cs_state and cs_side must be different streams of one device.
+ * Everything else as for lc_compress, with one restriction: the statistics pass hands the encode pass one byte
+ * per element, which identifies the bucket only while every |delta| < 2 (exponent field below 128). lc_compress
+ * falls back to reading base and cur again in that case; this call cannot, because it has released them, and
+ * reports LC_ERR_RANGE in the status word instead (the stream is then unusable; use lc_compress).
+ */
+int lc_compress_async(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                      uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs_state,
+                      lc_cuda_stream_t cs_side, lc_cuda_event_t state_read);
+
+/*
+ * Checkpoint merging (Section 3.2, "Checkpoint Merging"): the k streams that lead from `base` to a later tracked
+ * state become one super-step stream, so that a later recovery applies one stream instead of k.
+ * The paper does not say how the merged checkpoint is coded. The reading taken here is the scheme applied once more
+ * to the summed change:
+ *   merged <- LC(recover(base, streams) - base),
+ * i.e. lc_recover followed by lc_compress against the same base, in one call. The merged stream quantizes a second
+ * time: recovering it gives a state within the quantization error of, not bit-identical to, the state the k streams
+ * recover (their sum takes many more distinct values than one stream's buckets have representatives).
+ * base, streams, stream_bytes, k, n   as for lc_recover.
+ * nbits, stream, stream_capacity      as for lc_compress: the merged stream.
+ * scratch    DEVICE, n fp32, 16-byte aligned, written: receives recover(base, streams), which is also the state the
+ *            merged stream was coded from. Must not overlap base or the streams.
+ * workspace  as for lc_compress.
+ * Errors as for lc_recover and lc_compress (malformed input stream, non-finite merged delta, buffers too small).
+ */
+int lc_merge(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k, uint64_t n,
+             int nbits, void* stream, uint64_t stream_capacity, float* scratch, void* workspace,
+             uint64_t workspace_bytes, lc_cuda_stream_t cs);
 
 /* Copies a stream's header to the host. `stream` DEVICE, `info` HOST. Waits for `cs`. */
 int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs);

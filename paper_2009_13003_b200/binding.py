@@ -13,12 +13,12 @@ import torch
 
 from . import build as _build
 
-OK, ERR_ARG, ERR_CAPACITY, ERR_NONFINITE, ERR_FORMAT, ERR_MISMATCH, ERR_TIMEOUT, ERR_CUDA = 0, -1, -2, -3, -4, -5, -6, -7
+OK, ERR_ARG, ERR_CAPACITY, ERR_NONFINITE, ERR_FORMAT, ERR_MISMATCH, ERR_TIMEOUT, ERR_CUDA, ERR_RANGE = 0, -1, -2, -3, -4, -5, -6, -7, -8
 MAX_CHAIN = 8
 
 SYMBOLS = (
     "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_update", "lc_compress_timed",
-    "lc_recover", "lc_compress_opt", "lc_debug_compress_wait",
+    "lc_recover", "lc_compress_opt", "lc_debug_compress_wait", "lc_merge", "lc_compress_async",
     "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
     "lc_debug_bins", "lc_debug_codes", "lc_compress_noalloc",
 )
@@ -68,6 +68,8 @@ def lib():
     L.lc_debug_compress_wait.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, C.c_uint32, C.c_uint32, vp]
     L.lc_compress_timed.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, C.POINTER(C.c_float)]
     L.lc_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
+    L.lc_compress_async.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, vp, vp]
+    L.lc_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, vp, vp, u64, vp]
     L.lc_stream_info.argtypes = [vp, C.POINTER(LCInfo), vp]
     L.lc_last_status.argtypes = [vp, vp]
     L.lc_host_arena_bytes.argtypes = [u64, i32, i32]
@@ -221,6 +223,45 @@ def recover(base, streams, out=None, workspace=None):
     recover_async(base, streams, out, workspace)
     _check(last_status(workspace), "lc_recover (device)")
     return out
+
+
+def compress_two_streams(base, cur, nbits, stream, workspace, state_stream, side_stream, state_read):
+    """Enqueues lc_compress_async: the statistics pass on `state_stream` (torch.cuda.Stream), then `state_read`
+    (torch.cuda.Event) recorded there; table and encode on `side_stream` behind that event."""
+    _f32_cuda(base, "base"), _f32_cuda(cur, "cur")
+    if not state_read.cuda_event:  # torch creates the CUDA event at its first record
+        state_read.record(state_stream)
+    rc = lib().lc_compress_async(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(),
+                                 stream.numel(), workspace.data_ptr(), workspace.numel(),
+                                 C.c_void_p(state_stream.cuda_stream), C.c_void_p(side_stream.cuda_stream),
+                                 C.c_void_p(state_read.cuda_event))
+    _check(rc, "lc_compress_async")
+
+
+def merge_async(base, streams, nbits, stream, scratch, workspace):
+    """Enqueues lc_merge: the super-step stream of `streams` over `base` (Section 3.2, checkpoint merging)."""
+    _f32_cuda(base, "base"), _f32_cuda(scratch, "scratch")
+    k = len(streams)
+    ptrs = (C.c_void_p * k)(*[s.data_ptr() for s in streams])
+    sizes = (C.c_uint64 * k)(*[s.numel() for s in streams])
+    rc = lib().lc_merge(base.data_ptr(), ptrs, sizes, k, base.numel(), nbits, stream.data_ptr(), stream.numel(),
+                        scratch.data_ptr(), workspace.data_ptr(), workspace.numel(), _cs(base.device))
+    _check(rc, "lc_merge")
+
+
+def merge(base, streams, nbits, stream=None, scratch=None, workspace=None):
+    """One stream that stands for `streams` applied to `base`: compress(base, recover(base, streams)). Returns the
+    merged stream trimmed to its size; `scratch` (allocated if None) receives the recovered state."""
+    n = base.numel()
+    if stream is None:
+        stream = alloc_stream(n, nbits, base.device)
+    if scratch is None:
+        scratch = torch.empty_like(base)
+    if workspace is None:
+        workspace = alloc_workspace(n, base.device)
+    merge_async(base, streams, nbits, stream, scratch, workspace)
+    _check(last_status(workspace), "lc_merge (device)")
+    return stream[: stream_info(stream).total_bytes]
 
 
 def host_arena_bytes(n, nbits, k) -> int:

@@ -28,7 +28,7 @@ Carved carve(void* workspace, const WorkspaceLayout& W) {
 // lc_compress and lc_compress_update: argument checks, then memset + three kernels on `cs`.
 int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, void* stream, uint64_t stream_capacity,
                   float* tracked_out, void* workspace, uint64_t workspace_bytes, const EncodeOptions& opt,
-                  cudaStream_t cs) {
+                  cudaStream_t cs, bool keep_status = false) {
   if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
   if (!stream || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
   if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
@@ -37,11 +37,13 @@ int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, vo
   if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
   const Carved c = carve(workspace, W);
 
-  // control block and tile descriptors start at zero
-  cudaError_t e = cudaMemsetAsync(workspace, 0, W.plane_off, cs);
+  // control block and tile descriptors start at zero (keep_status: all but the status word, which holds the
+  // outcome of the pass that produced `cur`; the table pass then leaves the vector alone if it is set)
+  const uint64_t skip = keep_status ? sizeof(int32_t) : 0;
+  cudaError_t e = cudaMemsetAsync(static_cast<uint8_t*>(workspace) + skip, 0, W.plane_off - skip, cs);
   if (e != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, cs)) != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), tracked_out, opt,
                          cs)) != cudaSuccess)
     return LC_ERR_CUDA;
@@ -71,6 +73,7 @@ const char* lc_strerror(int code) {
     case LC_ERR_MISMATCH: return "element count mismatch";
     case LC_ERR_TIMEOUT: return "device-side wait timed out";
     case LC_ERR_CUDA: return "CUDA runtime error";
+    case LC_ERR_RANGE: return "a delta of magnitude 2 or more needs the state that the call has released";
     default: return "unknown status";
   }
 }
@@ -138,7 +141,7 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
   ok = ok && cudaEventRecord(ev[0], cs) == cudaSuccess;
   ok = ok && launch_stats(base, cur, n, c.ctl, c.plane, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[1], cs) == cudaSuccess;
-  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), cs) == cudaSuccess;
+  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[2], cs) == cudaSuccess;
   ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[3], cs) == cudaSuccess;
@@ -173,6 +176,47 @@ int lc_recover(const float* base, const void* const* streams, const uint64_t* st
     src = out;
   }
   return LC_OK;
+}
+
+int lc_compress_async(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                      uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs_state,
+                      lc_cuda_stream_t cs_side, lc_cuda_event_t state_read) {
+  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (!stream || !workspace || !state_read || cs_state == cs_side || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
+  if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
+    return LC_ERR_ARG;
+  const WorkspaceLayout W = workspace_layout(n);
+  if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
+  const Carved c = carve(workspace, W);
+  // on the stream that owns the model state: everything that reads it
+  if (cudaMemsetAsync(workspace, 0, W.plane_off, cs_state) != cudaSuccess) return LC_ERR_CUDA;
+  if (launch_stats(base, cur, n, c.ctl, c.plane, cs_state) != cudaSuccess) return LC_ERR_CUDA;
+  if (cudaEventRecord(state_read, cs_state) != cudaSuccess) return LC_ERR_CUDA;
+  // beside whatever cs_state does next: table and encode, which work on the bucket statistics and the key plane
+  if (cudaStreamWaitEvent(cs_side, state_read, 0) != cudaSuccess) return LC_ERR_CUDA;
+  if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), /*wide_ok=*/false, cs_side) != cudaSuccess)
+    return LC_ERR_CUDA;
+  if (launch_encode(c.ctl, c.tiles, c.plane, nullptr, nullptr, n, static_cast<uint8_t*>(stream), nullptr,
+                    EncodeOptions(), cs_side) != cudaSuccess)
+    return LC_ERR_CUDA;
+  return LC_OK;
+}
+
+int lc_merge(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k, uint64_t n,
+             int nbits, void* stream, uint64_t stream_capacity, float* scratch, void* workspace,
+             uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+  if (nbits < 1 || nbits > 8) return LC_ERR_ARG;
+  if (!stream || !aligned(stream, 16) || (n > 0 && (!scratch || !aligned(scratch, 16) || scratch == base)))
+    return LC_ERR_ARG;
+  if (workspace_bytes < workspace_layout(n).total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
+  // the state the k streams recover ...
+  int rc = lc_recover(base, streams, stream_bytes, k, n, scratch, workspace, workspace_bytes, cs);
+  if (rc != LC_OK) return rc;
+  // ... coded against the same base. The compress pass starts by clearing the status word, so a stream that the
+  // recovery rejected has to be remembered across it: the encode pass leaves, and the status stays, if the word
+  // was already set when the table pass looked (see compress_impl's `keep_status`).
+  return compress_impl(base, scratch, n, nbits, stream, stream_capacity, nullptr, workspace, workspace_bytes,
+                       EncodeOptions(), cs, /*keep_status=*/true);
 }
 
 int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {

@@ -120,7 +120,9 @@ struct EncodeOptions {
 // ---- launchers (each defined next to its kernel) ---------------------------------------------------
 cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
                          cudaStream_t cs);
-cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, cudaStream_t cs);
+// wide_ok: false if the encode pass will not be able to read base and cur (the table pass then rejects a vector
+// with an exponent field >= 128 with LC_ERR_RANGE)
+cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, cudaStream_t cs);
 // tracked_out: nullptr, or where to write base + quantized delta (may be base itself)
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
                           const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, const EncodeOptions& opt,

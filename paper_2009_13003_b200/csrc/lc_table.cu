@@ -20,7 +20,7 @@ __device__ __forceinline__ void store_le(uint8_t* p, uint64_t v, int bytes) {
 }
 
 __global__ void __launch_bounds__(kTableThreads)
-table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restrict__ stream) {
+table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restrict__ stream, int wide_ok) {
   __shared__ uint32_t warp_cand[16];
   __shared__ uint16_t sym_of_key[kKeys];
   __shared__ unsigned long long sym_count[kMaxSym];
@@ -39,6 +39,12 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
 
+  // ---- an earlier pass of the same call has failed (lc_merge: a stream was rejected): leave no stream behind
+  if (ctl->status != 0) {  // nothing in this kernel has written the word yet: the same for every thread
+    if (tid < 64) stream[tid] = 0;
+    return;
+  }
+
   // ---- non-finite deltas make the vector unencodable ------------------------------------------
   const bool bad = (tid == 255 || tid == 511) && ctl->count[tid] != 0;
   if (__syncthreads_or(bad)) {
@@ -52,6 +58,14 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   // ---- does the one-byte key plane identify every bucket? (only if all exponent fields are < 128)
   const bool big = (tid & 255) >= 128 && ctl->count[tid] != 0;
   const int wide = __syncthreads_or(big);
+  if (wide && !wide_ok) {
+    // the caller has released base and cur, and the one-byte keys do not identify the buckets of this vector
+    if (tid == 0) {
+      set_status(&ctl->status, LC_ERR_RANGE);
+      for (int b = 0; b < 64; ++b) stream[b] = 0;
+    }
+    return;
+  }
 
   // ---- priority promotion -------------------------------------------------------------------------
   // thread `tid` < 508 looks at the key of priority position tid: exponent descending, + before -.
@@ -235,8 +249,8 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
 
 }  // namespace
 
-cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, cudaStream_t cs) {
-  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream);
+cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, cudaStream_t cs) {
+  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0);
   return cudaGetLastError();
 }
 
