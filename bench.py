@@ -328,15 +328,21 @@ def run_ours(args, rank, world, local_rank):
     out = torch.empty_like(u0)
     stream_bytes = [int(s.numel()) for s in streams]
     torch.cuda.synchronize()
-    # size of the last snapshot under the paper's three stages (Section 4.3: E, E+P, E+P+H), as fractions of
-    # the full fp32 state; the first two by the paper's size model n*ceil(log2 k) + k*32 bits
+    # size of the last snapshot under the paper's three stages (Section 4.3: E, E+P, E+P+H) as fractions of the full
+    # fp32 state: measured on real streams (fixed-width indices with every bucket kept; fixed-width indices after
+    # promotion; Huffman-coded), and beside them the paper's size model n*ceil(log2 k) + k*32 bits
     count, _, _ = lc.debug_bins(ws)
     k_e = int((count > 0).sum())
     nsym = int(lc.stream_info(streams[-1]).nsym)
     width = lambda k: max(1, (k - 1).bit_length())
+    sbuf_e = lc.alloc_stream(n, 9, dev)
+    bytes_e = int(lc.compress(tracked, u, 9, stream=sbuf_e, workspace=ws, fixed=True).numel())
+    bytes_ep = int(lc.compress(tracked, u, nbits, stream=sbuf_e, workspace=ws, fixed=True).numel())
+    del sbuf_e
     size_model = {"occupied_buckets": k_e, "kept_symbols": nsym,
-                  "E": (n * width(k_e) + 32 * k_e) / (32.0 * n), "E+P": (n * width(nsym) + 32 * nsym) / (32.0 * n),
-                  "E+P+H": 8.0 * stream_bytes[-1] / (32.0 * n)}
+                  "E": bytes_e / (4.0 * n), "E+P": bytes_ep / (4.0 * n), "E+P+H": stream_bytes[-1] / (4.0 * n),
+                  "model_E": (n * width(k_e) + 32 * k_e) / (32.0 * n),
+                  "model_E+P": (n * width(nsym) + 32 * nsym) / (32.0 * n)}
 
     def step():
         lc.compress_async(tracked, u, nbits, sbuf, ws)
@@ -404,6 +410,49 @@ def run_ours(args, rank, world, local_rank):
     assert lc.last_status(ws) == 0
     assert torch.equal(sbuf[: stream_bytes[-1]], streams[-1]), "fused compress did not reproduce the stream"
     recover_chain(out)  # `out` holds the whole chain's result again
+    # ---- asynchronous execution (Section 3.2): statistics pass on the stream that owns the state, table and encode
+    # on a side stream, beside a synthetic "next training iteration" (bf16 matrix products on the state's stream);
+    # outside the timed region. exposed = what the state's stream waits for before its next work can start.
+    state_s, side_s = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ev_read = torch.cuda.Event()
+    ma = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+    mb = torch.randn(8192, 8192, device=dev, dtype=torch.bfloat16)
+    mc = torch.empty_like(ma)
+
+    def next_iteration():
+        for _ in range(3):
+            torch.matmul(ma, mb, out=mc)
+
+    asy = {"exposed": [], "overlapped": [], "serial": [], "work": []}
+    for it in range(5):
+        torch.cuda.synchronize()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        with torch.cuda.stream(state_s):
+            e[0].record()
+            lc.compress_two_streams(tracked, u, nbits, sbuf, ws, state_s, side_s, ev_read)
+            e[1].record()
+            next_iteration()
+            e[2].record()
+            state_s.wait_stream(side_s)
+            e[3].record()
+        torch.cuda.synchronize()
+        assert lc.last_status(ws) == 0
+        f = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        with torch.cuda.stream(state_s):
+            f[0].record()
+            lc.compress_async(tracked, u, nbits, sbuf, ws)
+            f[1].record()
+            next_iteration()
+            f[2].record()
+        torch.cuda.synchronize()
+        if it >= 1:
+            asy["exposed"].append(e[0].elapsed_time(e[1]))
+            asy["overlapped"].append(e[0].elapsed_time(e[3]))
+            asy["serial"].append(f[0].elapsed_time(f[2]))
+            asy["work"].append(f[1].elapsed_time(f[2]))
+    assert torch.equal(sbuf[: stream_bytes[-1]], streams[-1]), "two-stream compress did not reproduce the stream"
+    asy = {k: statistics.median(v) for k, v in asy.items()}
+    del ma, mb, mc
     # ---- checkpoint merging (Section 3.2): the chain as one super-step stream; outside the timed region
     merge_ms = merged_bytes = None
     if chain <= lc.MAX_CHAIN:
@@ -503,6 +552,10 @@ def run_ours(args, rank, world, local_rank):
             "ms": merge_ms, "streams_in": chain, "merged_ratio": 4.0 * n / merged_bytes,
             "alg_gbs": (4.0 * n + sum(stream_bytes) + merged_bytes) / (merge_ms * 1e-3) / 1e9,
             "frac_of_peak": (4.0 * n + sum(stream_bytes) + merged_bytes) / (merge_ms * 1e-3) / 1e9 / peak},
+        # lc_compress_async beside a synthetic next iteration (3 bf16 products of 8192^2 matrices on the state's
+        # stream): exposed = memset + statistics pass; overlapped / serial = both finished, two streams / one
+        "async": {"exposed_ms": asy["exposed"], "next_iteration_ms": asy["work"], "overlapped_ms": asy["overlapped"],
+                  "serial_ms": asy["serial"]},
         "ratio": {"stream": 4.0 * n / stream_bytes[-1], "bits_per_element": 8.0 * sbar[-1],
                   "code_bits_per_element": code_bits, "entropy_bits_per_element": entropy_bits},
         "size_model": size_model,

@@ -29,7 +29,7 @@ extern "C" {
 #endif
 
 #define LC_OK 0
-#define LC_ERR_ARG (-1)       /* null / misaligned pointer, nbits outside 1..8, k outside 1..LC_MAX_CHAIN, n >= 2^32 */
+#define LC_ERR_ARG (-1)       /* null / misaligned pointer, nbits outside 1..9, k outside 1..LC_MAX_CHAIN, n >= 2^32 */
 #define LC_ERR_CAPACITY (-2)  /* stream or workspace buffer too small */
 #define LC_ERR_NONFINITE (-3) /* some delta is Inf or NaN; the stream must not be used */
 #define LC_ERR_FORMAT (-4)    /* malformed stream */
@@ -55,6 +55,7 @@ typedef struct lc_info {
   uint32_t max_len;        /* longest code */
   uint32_t nchunks;
   int32_t valid;           /* 1 if magic, version and constants are those of format version 1 */
+  uint32_t fixed_width;    /* 1 if the stream carries fixed-width codes (format section 1.5) */
 } lc_info;
 
 /* Library version (major*100 + minor). */
@@ -81,7 +82,8 @@ uint64_t lc_workspace_bytes(uint64_t n);
  *   are Huffman-coded.
  * base, cur   DEVICE, read-only, n contiguous fp32 each, 16-byte aligned.
  * n           number of elements, 0 <= n < 2^32.
- * nbits       x of the x-bit priority promotion, 1..8.
+ * nbits       x of the x-bit priority promotion, 1..9 (9 keeps every occupied bucket: exponent-based
+ *             quantization alone, the "E" stage of Section 4.3).
  * stream      DEVICE, written; 16-byte aligned; stream_capacity >= lc_stream_bound(n, nbits).
  *             The stream's size is in its header (lc_stream_info).
  * workspace   DEVICE scratch, 256-byte aligned, workspace_bytes >= lc_workspace_bytes(n). Its contents
@@ -110,17 +112,22 @@ int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbit
                        lc_cuda_stream_t cs);
 
 /*
- * lc_compress / lc_compress_update with options (the same passages; `options` only changes how the work is
- * scheduled, never a byte of the result).
+ * lc_compress / lc_compress_update with options (the same passages).
  * tracked_out   NULL for lc_compress's behaviour, else as for lc_compress_update.
- * options       0, or LC_OPT_NO_DEVICE_WAIT: the byte offsets of the chunks (format section 3.3) come from a
+ * options       0, or a combination of:
+ *               LC_OPT_NO_DEVICE_WAIT: the byte offsets of the chunks (format section 3.3) come from a
  *               sizes pass and a one-CTA prefix-sum kernel instead of the decoupled look-back between running
  *               CTAs of the encode pass. No kernel of the call then ever waits for another CTA, so
  *               LC_ERR_TIMEOUT cannot occur; the price is one more pass over the one-byte key plane.
  *               For deployments where a device-side spin, however bounded, is not acceptable.
+ *               LC_OPT_FIXED_WIDTH: the bucket indices are written with ceil(log2 nsym) bits each instead of their
+ *               Huffman codes (format section 1.5): the stream of Section 3.1.1's size model, n*ceil(log2 k) bits
+ *               of indices, and the "E" (with nbits 9) and "E+P" stages of Section 4.3's size breakdown as real
+ *               streams. lc_recover reads such streams like any other. This option does change the bytes.
  * Any other bit in `options` returns LC_ERR_ARG.
  */
 #define LC_OPT_NO_DEVICE_WAIT 1u
+#define LC_OPT_FIXED_WIDTH 2u
 int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                     uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
                     uint32_t options, lc_cuda_stream_t cs);

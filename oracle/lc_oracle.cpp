@@ -42,6 +42,8 @@ constexpr uint64_t kLanes = 32;         // lane sub-streams per chunk
 constexpr uint64_t kGroup = 4;          // consecutive elements a lane takes per step
 constexpr uint64_t kSteps = kChunkElems / (kLanes * kGroup);
 
+typedef uint16_t sym_t;  // symbol ids reach 508 when every bucket is kept (nbits = 9)
+
 uint32_t float_bits(float f) {
   uint32_t u;
   std::memcpy(&u, &f, sizeof u);
@@ -89,7 +91,7 @@ void delta_buckets(const float* base, const float* cur, uint64_t n, Bucket* buck
 
 struct Selection {
   int nsym = 1;                 // K + 1
-  int key_of_symbol[256] = {};  // key_of_symbol[0] is 0 by convention
+  int key_of_symbol[512] = {};  // key_of_symbol[0] is 0 by convention
   int symbol_of_key[512] = {};  // 0 for everything that is not kept
 };
 
@@ -192,15 +194,16 @@ struct Table {
   int nbits = 0;
   int nsym = 1;
   int max_len = 0;
-  int key[256] = {};
-  int len[256] = {};
-  float rep[256] = {};
-  uint64_t count[256] = {};
-  uint64_t code[256] = {};
+  int fixed = 0;  // 1: fixed-width codes (format section 1.5) instead of the Huffman code
+  int key[512] = {};
+  int len[512] = {};
+  float rep[512] = {};
+  uint64_t count[512] = {};
+  uint64_t code[512] = {};
 };
 
 // Steps of Sections 3.1.1-3.1.2 that turn bucket statistics into the symbol table.
-int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selection* sel_out) {
+int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selection* sel_out, int fixed = 0) {
   for (int s = 0; s <= 1; ++s)
     if (buckets[256 * s + 255].count > 0) return LCO_ERR_NONFINITE;
   const Selection sel = priority_promotion(buckets, nbits);
@@ -218,8 +221,19 @@ int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selectio
   t->key[0] = 0;
   t->rep[0] = 0.0f;
   t->count[0] = n - kept_total;
-  huffman_lengths(t->count, t->nsym, t->len);
-  canonical_codes(t->len, t->nsym, t->code);
+  t->fixed = fixed;
+  if (fixed) {
+    // Section 3.1.1's size model: every bucket index takes ceil(log2 k) bits; the code of a symbol is its id.
+    int width = 0;
+    while ((1 << width) < t->nsym) width += 1;
+    for (int j = 0; j < t->nsym; ++j) {
+      t->len[j] = width;
+      t->code[j] = static_cast<uint64_t>(j);
+    }
+  } else {
+    huffman_lengths(t->count, t->nsym, t->len);
+    canonical_codes(t->len, t->nsym, t->code);
+  }
   for (int j = 0; j < t->nsym; ++j) t->max_len = std::max(t->max_len, t->len[j]);
   if (sel_out) *sel_out = sel;
   return LCO_OK;
@@ -319,7 +333,8 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   if (!(s[0] == 'L' && s[1] == 'C' && s[2] == 'C' && s[3] == '1')) return LCO_ERR_FORMAT;
   if (get_le(s + 4, 2) != 1) return LCO_ERR_FORMAT;
   const int nbits = static_cast<int>(s[6]);
-  if (nbits < 1 || nbits > 8 || s[7] != 0) return LCO_ERR_FORMAT;
+  if (nbits < 1 || nbits > 9 || s[7] > 1) return LCO_ERR_FORMAT;
+  const int fixed = static_cast<int>(s[7]);
   const uint64_t n = get_le(s + 8, 8);
   const uint64_t nsym = get_le(s + 16, 4);
   const uint64_t max_len = get_le(s + 20, 4);
@@ -350,7 +365,7 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
     p.table.rep[j] = bits_float(static_cast<uint32_t>(get_le(e + 4, 4)));
     p.table.count[j] = get_le(e + 8, 8);
     if (e[3] != 0 || p.table.len[j] > 63) return LCO_ERR_FORMAT;
-    if (p.table.count[j] == 0 && p.table.len[j] != 0) return LCO_ERR_FORMAT;
+    if (!fixed && p.table.count[j] == 0 && p.table.len[j] != 0) return LCO_ERR_FORMAT;
     if (p.table.count[j] > 0) used += 1;
     count_sum += p.table.count[j];
     bit_sum += p.table.count[j] * static_cast<uint64_t>(p.table.len[j]);
@@ -359,7 +374,15 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   if (count_sum != n || bit_sum != payload_bits || static_cast<uint64_t>(seen_max) != max_len)
     return LCO_ERR_FORMAT;
   p.table.max_len = seen_max;
-  if (used >= 2) {
+  p.table.fixed = fixed;
+  if (fixed) {
+    int width = 0;
+    while ((1ull << width) < nsym) width += 1;
+    for (uint64_t j = 0; j < nsym; ++j) {
+      if (p.table.len[j] != width) return LCO_ERR_FORMAT;
+      p.table.code[j] = j;
+    }
+  } else if (used >= 2) {
     // Kraft equality, as an exact integer sum of 2^(63-len).
     unsigned __int128 kraft = 0;
     for (uint64_t j = 0; j < nsym; ++j) {
@@ -371,7 +394,7 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   } else if (seen_max != 0) {
     return LCO_ERR_FORMAT;
   }
-  canonical_codes(p.table.len, p.table.nsym, p.table.code);
+  if (!fixed) canonical_codes(p.table.len, p.table.nsym, p.table.code);
 
   // chunk index must start at 0, be non-decreasing, 16-aligned and end at the payload size.
   const uint8_t* ci = s + L.chunk_index_off;
@@ -419,7 +442,7 @@ int build_tree(const Table& t, CodeTree* tree) {
 }
 
 // Decodes the symbols of chunk c by walking the code tree one bit at a time.
-int decode_chunk(const uint8_t* s, const Parsed& p, const CodeTree& tree, uint64_t c, uint8_t* sym /*[n]*/) {
+int decode_chunk(const uint8_t* s, const Parsed& p, const CodeTree& tree, uint64_t c, sym_t* sym /*[n]*/) {
   const Layout& L = p.layout;
   const uint8_t* chunk_index = s + L.chunk_index_off;
   const uint8_t* lane_index = s + L.lane_index_off;
@@ -444,7 +467,7 @@ int decode_chunk(const uint8_t* s, const Parsed& p, const CodeTree& tree, uint64
           if (node < 0) break;
           if (node == 0) return LCO_ERR_FORMAT;
         }
-        sym[i] = static_cast<uint8_t>(-node - 1);
+        sym[i] = static_cast<sym_t>(-node - 1);
       }
     }
     if (bit != lane_end) return LCO_ERR_FORMAT;
@@ -453,13 +476,13 @@ int decode_chunk(const uint8_t* s, const Parsed& p, const CodeTree& tree, uint64
 }
 
 // Decodes every symbol of a stream, chunk after chunk.
-int decode_symbols(const uint8_t* s, uint64_t bytes, const Parsed& p, uint8_t* sym /*[n]*/) {
+int decode_symbols(const uint8_t* s, uint64_t bytes, const Parsed& p, sym_t* sym /*[n]*/) {
   (void)bytes;
   CodeTree tree;
   const int rc = build_tree(p.table, &tree);
   if (rc != LCO_OK) return rc;
   if (p.table.max_len == 0) {
-    for (uint64_t i = 0; i < p.n; ++i) sym[i] = static_cast<uint8_t>(tree.only);
+    for (uint64_t i = 0; i < p.n; ++i) sym[i] = static_cast<sym_t>(tree.only);
     return LCO_OK;
   }
   for (uint64_t c = 0; c < p.layout.nchunks; ++c) {
@@ -484,7 +507,7 @@ void write_header_and_table(uint8_t* stream, const Table& t, uint64_t n, int nbi
   h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
   put_le(h + 4, 1, 2);
   h[6] = static_cast<uint8_t>(nbits);
-  h[7] = 0;
+  h[7] = static_cast<uint8_t>(t.fixed);
   put_le(h + 8, n, 8);
   put_le(h + 16, static_cast<uint64_t>(t.nsym), 4);
   put_le(h + 20, static_cast<uint64_t>(t.max_len), 4);
@@ -534,13 +557,14 @@ int lco_bins(const float* base, const float* cur, uint64_t n, uint64_t* count, u
 
 // Symbol table (selection, representatives, counts, code lengths, codes) for a delta vector.
 // Arrays have 256 entries; returns nsym (>= 1) or a negative status.
-int lco_table(const float* base, const float* cur, uint64_t n, int nbits, int* key, float* rep,
-              uint64_t* count, int* len, uint64_t* code) {
-  if (nbits < 1 || nbits > 8) return LCO_ERR_ARG;
+// `fixed`: 0 for the Huffman code, 1 for fixed-width codes (format section 1.5).
+int lco_table_mode(const float* base, const float* cur, uint64_t n, int nbits, int fixed, int* key, float* rep,
+                   uint64_t* count, int* len, uint64_t* code) {
+  if (nbits < 1 || nbits > 9 || fixed < 0 || fixed > 1) return LCO_ERR_ARG;
   std::vector<Bucket> buckets(512);
   delta_buckets(base, cur, n, buckets.data());
   Table t;
-  const int rc = build_table(buckets.data(), n, nbits, &t, nullptr);
+  const int rc = build_table(buckets.data(), n, nbits, &t, nullptr, fixed);
   if (rc != LCO_OK) return rc;
   for (int j = 0; j < t.nsym; ++j) {
     key[j] = t.key[j];
@@ -552,16 +576,21 @@ int lco_table(const float* base, const float* cur, uint64_t n, int nbits, int* k
   return t.nsym;
 }
 
+int lco_table(const float* base, const float* cur, uint64_t n, int nbits, int* key, float* rep,
+              uint64_t* count, int* len, uint64_t* code) {
+  return lco_table_mode(base, cur, n, nbits, 0, key, rep, count, len, code);
+}
+
 // Per-element symbol ids of the quantized delta (what the payload encodes), in element order.
-int lco_symbols(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* sym) {
-  if (nbits < 1 || nbits > 8) return LCO_ERR_ARG;
+int lco_symbols(const float* base, const float* cur, uint64_t n, int nbits, uint16_t* sym) {
+  if (nbits < 1 || nbits > 9) return LCO_ERR_ARG;
   std::vector<Bucket> buckets(512);
   delta_buckets(base, cur, n, buckets.data());
   Table t;
   Selection sel;
   const int rc = build_table(buckets.data(), n, nbits, &t, &sel);
   if (rc != LCO_OK) return rc;
-  for (uint64_t i = 0; i < n; ++i) sym[i] = static_cast<uint8_t>(sel.symbol_of_key[bucket_key(cur[i] - base[i])]);
+  for (uint64_t i = 0; i < n; ++i) sym[i] = static_cast<sym_t>(sel.symbol_of_key[bucket_key(cur[i] - base[i])]);
   return LCO_OK;
 }
 
@@ -587,15 +616,17 @@ uint64_t lco_model_bits(uint64_t n, uint64_t k, uint64_t b) {
 uint64_t lco_stream_bound(uint64_t n, int nbits) { return stream_bound(n, nbits); }
 
 // Full compress pass: Algorithm 1 steps 4-6. Writes the stream, returns its size through *out_bytes.
-int lco_compress(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* stream,
-                 uint64_t capacity, uint64_t* out_bytes) {
-  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LCO_ERR_ARG;
+// `fixed`: 0 for the Huffman code (Section 3.1.2), 1 for fixed-width bucket indices (the size model of
+// Section 3.1.1 and the "E" / "E+P" stages of Section 4.3's size breakdown).
+int lco_compress_mode(const float* base, const float* cur, uint64_t n, int nbits, int fixed, uint8_t* stream,
+                      uint64_t capacity, uint64_t* out_bytes) {
+  if (nbits < 1 || nbits > 9 || fixed < 0 || fixed > 1 || n >= (1ull << 32)) return LCO_ERR_ARG;
   if (capacity < stream_bound(n, nbits)) return LCO_ERR_CAPACITY;
   std::vector<Bucket> buckets(512);
   delta_buckets(base, cur, n, buckets.data());
   Table t;
   Selection sel;
-  const int rc = build_table(buckets.data(), n, nbits, &t, &sel);
+  const int rc = build_table(buckets.data(), n, nbits, &t, &sel, fixed);
   if (rc != LCO_OK) return rc;
 
   const Layout L = layout_for(n, t.nsym);
@@ -620,8 +651,13 @@ int lco_compress(const float* base, const float* cur, uint64_t n, int nbits, uin
   return LCO_OK;
 }
 
+int lco_compress(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* stream,
+                 uint64_t capacity, uint64_t* out_bytes) {
+  return lco_compress_mode(base, cur, n, nbits, 0, stream, capacity, out_bytes);
+}
+
 // Symbol ids stored in a stream, in element order (decode only, no arithmetic).
-int lco_decode_symbols(const uint8_t* stream, uint64_t bytes, uint64_t n, uint8_t* sym) {
+int lco_decode_symbols(const uint8_t* stream, uint64_t bytes, uint64_t n, uint16_t* sym) {
   Parsed p;
   const int rc = parse_stream(stream, bytes, &p);
   if (rc != LCO_OK) return rc;
@@ -641,7 +677,7 @@ int lco_recover(const float* base, const uint8_t* const* streams, const uint64_t
     if (parsed[j].n != n) return LCO_ERR_MISMATCH;
   }
   std::vector<float> x(base, base + n);
-  std::vector<uint8_t> sym(n);
+  std::vector<sym_t> sym(n);
   for (int j = 0; j < k; ++j) {
     const int rc = decode_symbols(streams[j], stream_bytes[j], parsed[j], sym.data());
     if (rc != LCO_OK) return rc;
@@ -653,7 +689,7 @@ int lco_recover(const float* base, const uint8_t* const* streams, const uint64_t
 
 // Algorithm 1 step 7 computed directly, without a bitstream: out = base + quantized(cur - base).
 int lco_apply_quantized(const float* base, const float* cur, uint64_t n, int nbits, float* out) {
-  if (nbits < 1 || nbits > 8) return LCO_ERR_ARG;
+  if (nbits < 1 || nbits > 9) return LCO_ERR_ARG;
   std::vector<Bucket> buckets(512);
   delta_buckets(base, cur, n, buckets.data());
   Table t;
@@ -669,7 +705,7 @@ int lco_apply_quantized(const float* base, const float* cur, uint64_t n, int nbi
 // payload + m*stride. Lets a test check chunks of a vector too large to code in full.
 int lco_compress_chunks(const float* base, const float* cur, uint64_t n, int nbits, const uint64_t* chunk_ids,
                         uint64_t m, uint16_t* lane_bits, uint8_t* payload, uint64_t stride, uint64_t* bytes) {
-  if (nbits < 1 || nbits > 8) return LCO_ERR_ARG;
+  if (nbits < 1 || nbits > 9) return LCO_ERR_ARG;
   std::vector<Bucket> buckets(512);
   delta_buckets(base, cur, n, buckets.data());
   Table t;
@@ -711,9 +747,9 @@ int lco_merge(const float* base, const uint8_t* const* streams, const uint64_t* 
 // and decoded independently once the table is known. The results are byte-identical to the
 // single-threaded functions (a test checks that).
 
-int lco_compress_mt(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* stream,
-                    uint64_t capacity, uint64_t* out_bytes, int nthreads) {
-  if (nbits < 1 || nbits > 8 || n >= (1ull << 32) || nthreads < 1) return LCO_ERR_ARG;
+int lco_compress_mode_mt(const float* base, const float* cur, uint64_t n, int nbits, int fixed, uint8_t* stream,
+                         uint64_t capacity, uint64_t* out_bytes, int nthreads) {
+  if (nbits < 1 || nbits > 9 || fixed < 0 || fixed > 1 || n >= (1ull << 32) || nthreads < 1) return LCO_ERR_ARG;
   if (capacity < stream_bound(n, nbits)) return LCO_ERR_CAPACITY;
   const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
   auto range = [&](int t, uint64_t total) {
@@ -742,7 +778,7 @@ int lco_compress_mt(const float* base, const float* cur, uint64_t n, int nbits, 
     }
   Table t;
   Selection sel;
-  const int rc = build_table(buckets.data(), n, nbits, &t, &sel);
+  const int rc = build_table(buckets.data(), n, nbits, &t, &sel, fixed);
   if (rc != LCO_OK) return rc;
   const Layout L = layout_for(n, t.nsym);
   std::memset(stream, 0, L.payload_off);
@@ -772,6 +808,11 @@ int lco_compress_mt(const float* base, const float* cur, uint64_t n, int nbits, 
   return LCO_OK;
 }
 
+int lco_compress_mt(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* stream,
+                    uint64_t capacity, uint64_t* out_bytes, int nthreads) {
+  return lco_compress_mode_mt(base, cur, n, nbits, 0, stream, capacity, out_bytes, nthreads);
+}
+
 int lco_recover_mt(const float* base, const uint8_t* const* streams, const uint64_t* stream_bytes, int k,
                    uint64_t n, float* out, int nthreads) {
   if (k < 1 || nthreads < 1) return LCO_ERR_ARG;
@@ -784,7 +825,7 @@ int lco_recover_mt(const float* base, const uint8_t* const* streams, const uint6
     if ((rc = build_tree(parsed[j].table, &trees[j])) != LCO_OK) return rc;
   }
   const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
-  std::vector<uint8_t> sym(n);
+  std::vector<sym_t> sym(n);
   std::vector<int> status(nthreads, LCO_OK);
   for (uint64_t i = 0; i < n; ++i) out[i] = base[i];
   for (int j = 0; j < k; ++j) {
@@ -793,7 +834,7 @@ int lco_recover_mt(const float* base, const uint8_t* const* streams, const uint6
       for (uint64_t c = c0; c < c1; ++c) {
         const uint64_t lo = c * kChunkElems, hi = std::min(n, lo + kChunkElems);
         if (parsed[j].table.max_len == 0) {
-          for (uint64_t i = lo; i < hi; ++i) sym[i] = static_cast<uint8_t>(trees[j].only);
+          for (uint64_t i = lo; i < hi; ++i) sym[i] = static_cast<sym_t>(trees[j].only);
         } else {
           const int rc = decode_chunk(streams[j], parsed[j], trees[j], c, sym.data());
           if (rc != LCO_OK) status[th] = rc;

@@ -35,6 +35,9 @@ def lib():
         L.lco_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp]
         L.lco_apply_quantized.argtypes = [vp, vp, u64, i32, vp]
         L.lco_compress_chunks.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
+        L.lco_table_mode.argtypes = [vp, vp, u64, i32, i32, vp, vp, vp, vp, vp]
+        L.lco_compress_mode.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64)]
+        L.lco_compress_mode_mt.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64), i32]
         L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_mt.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), i32]
         L.lco_recover_mt.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, i32]
@@ -64,17 +67,17 @@ def bins(base, cur):
     return count, mmin, mmax
 
 
-def table(base, cur, nbits):
-    """dict(key, rep, count, len, code), each of length nsym."""
+def table(base, cur, nbits, fixed=False):
+    """dict(key, rep, count, len, code), each of length nsym. ``fixed``: fixed-width codes instead of Huffman."""
     base, pb = _f32(base)
     cur, pc = _f32(cur)
-    key = np.zeros(256, np.int32)
-    rep = np.zeros(256, np.float32)
-    count = np.zeros(256, np.uint64)
-    ln = np.zeros(256, np.int32)
-    code = np.zeros(256, np.uint64)
-    rc = lib().lco_table(pb, pc, base.size, nbits, key.ctypes.data, rep.ctypes.data, count.ctypes.data,
-                         ln.ctypes.data, code.ctypes.data)
+    key = np.zeros(512, np.int32)
+    rep = np.zeros(512, np.float32)
+    count = np.zeros(512, np.uint64)
+    ln = np.zeros(512, np.int32)
+    code = np.zeros(512, np.uint64)
+    rc = lib().lco_table_mode(pb, pc, base.size, nbits, int(bool(fixed)), key.ctypes.data, rep.ctypes.data,
+                              count.ctypes.data, ln.ctypes.data, code.ctypes.data)
     if rc < 0:
         raise OracleError(rc)
     return dict(key=key[:rc], rep=rep[:rc], count=count[:rc], len=ln[:rc], code=code[:rc])
@@ -83,7 +86,7 @@ def table(base, cur, nbits):
 def symbols(base, cur, nbits):
     base, pb = _f32(base)
     cur, pc = _f32(cur)
-    sym = np.zeros(base.size, np.uint8)
+    sym = np.zeros(base.size, np.uint16)
     rc = lib().lco_symbols(pb, pc, base.size, nbits, sym.ctypes.data)
     if rc < 0:
         raise OracleError(rc)
@@ -112,20 +115,22 @@ def stream_bound(n, nbits):
     return int(lib().lco_stream_bound(n, nbits))
 
 
-def compress(base, cur, nbits, threads=None):
+def compress(base, cur, nbits, threads=None, fixed=False):
     """Returns the stream as a uint8 numpy array. ``threads``: None for the plain single-threaded pass, else the
-    number of host threads of the chunk-parallel timing mode (same bytes)."""
+    number of host threads of the chunk-parallel timing mode (same bytes). ``fixed``: fixed-width bucket indices
+    instead of the Huffman code. ``nbits`` 1...9 (9 keeps every bucket)."""
     base, pb = _f32(base)
     cur, pc = _f32(cur)
-    if not 1 <= nbits <= 8:
+    if not 1 <= nbits <= 9:
         raise OracleError(ERR_ARG)
     cap = stream_bound(base.size, nbits)
     buf = np.zeros(cap, np.uint8)
     out = C.c_uint64(0)
     if threads is None:
-        rc = lib().lco_compress(pb, pc, base.size, nbits, buf.ctypes.data, cap, C.byref(out))
+        rc = lib().lco_compress_mode(pb, pc, base.size, nbits, int(bool(fixed)), buf.ctypes.data, cap, C.byref(out))
     else:
-        rc = lib().lco_compress_mt(pb, pc, base.size, nbits, buf.ctypes.data, cap, C.byref(out), int(threads))
+        rc = lib().lco_compress_mode_mt(pb, pc, base.size, nbits, int(bool(fixed)), buf.ctypes.data, cap,
+                                        C.byref(out), int(threads))
     if rc < 0:
         raise OracleError(rc)
     return buf[: out.value].copy()
@@ -133,7 +138,7 @@ def compress(base, cur, nbits, threads=None):
 
 def decode_symbols(stream, n):
     stream = np.ascontiguousarray(stream, dtype=np.uint8)
-    sym = np.zeros(n, np.uint8)
+    sym = np.zeros(n, np.uint16)
     rc = lib().lco_decode_symbols(stream.ctypes.data, stream.size, n, sym.ctypes.data)
     if rc < 0:
         raise OracleError(rc)
@@ -163,7 +168,7 @@ def merge(base, streams, nbits):
     k = len(streams)
     ptrs = (C.c_void_p * k)(*[s.ctypes.data for s in streams])
     sizes = (C.c_uint64 * k)(*[s.size for s in streams])
-    if not 1 <= nbits <= 8:
+    if not 1 <= nbits <= 9:
         raise OracleError(ERR_ARG)
     cap = stream_bound(base.size, nbits)
     buf = np.zeros(cap, np.uint8)

@@ -29,7 +29,7 @@ class LCInfo(C.Structure):
     _fields_ = [
         ("n", C.c_uint64), ("total_bytes", C.c_uint64), ("payload_bits", C.c_uint64),
         ("payload_offset", C.c_uint64), ("nbits", C.c_uint32), ("nsym", C.c_uint32),
-        ("max_len", C.c_uint32), ("nchunks", C.c_uint32), ("valid", C.c_int32),
+        ("max_len", C.c_uint32), ("nchunks", C.c_uint32), ("valid", C.c_int32), ("fixed_width", C.c_uint32),
     ]
 
 
@@ -137,6 +137,7 @@ def compress_update_async(base, cur, nbits, stream, tracked_out, workspace):
 
 
 OPT_NO_DEVICE_WAIT = 1
+OPT_FIXED_WIDTH = 2
 
 
 def compress_opt_async(base, cur, nbits, stream, workspace, options, tracked_out=None):
@@ -175,14 +176,18 @@ def stream_info(stream) -> LCInfo:
     return info
 
 
-def compress(base, cur, nbits, stream=None, workspace=None):
-    """stream <- LC(cur - base). Returns the stream trimmed to its size (a view of ``stream``)."""
+def compress(base, cur, nbits, stream=None, workspace=None, fixed=False):
+    """stream <- LC(cur - base). Returns the stream trimmed to its size (a view of ``stream``). ``fixed``: fixed-width
+    bucket indices instead of the Huffman code (LC_OPT_FIXED_WIDTH)."""
     n = base.numel()
     if stream is None:
         stream = alloc_stream(n, nbits, base.device)
     if workspace is None:
         workspace = alloc_workspace(n, base.device)
-    compress_async(base, cur, nbits, stream, workspace)
+    if fixed:
+        compress_opt_async(base, cur, nbits, stream, workspace, OPT_FIXED_WIDTH)
+    else:
+        compress_async(base, cur, nbits, stream, workspace)
     _check(last_status(workspace), "lc_compress (device)")
     info = stream_info(stream)
     return stream[: info.total_bytes]

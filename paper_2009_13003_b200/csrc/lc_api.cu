@@ -29,7 +29,7 @@ Carved carve(void* workspace, const WorkspaceLayout& W) {
 int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, void* stream, uint64_t stream_capacity,
                   float* tracked_out, void* workspace, uint64_t workspace_bytes, const EncodeOptions& opt,
                   cudaStream_t cs, bool keep_status = false) {
-  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (nbits < 1 || nbits > kMaxNbits || n >= (1ull << 32)) return LC_ERR_ARG;
   if (!stream || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
   if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
     return LC_ERR_ARG;
@@ -43,7 +43,7 @@ int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, vo
   cudaError_t e = cudaMemsetAsync(static_cast<uint8_t*>(workspace) + skip, 0, W.plane_off - skip, cs);
   if (e != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, opt.fixed_width, cs)) != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), tracked_out, opt,
                          cs)) != cudaSuccess)
     return LC_ERR_CUDA;
@@ -79,7 +79,7 @@ const char* lc_strerror(int code) {
 }
 
 uint64_t lc_stream_bound(uint64_t n, int nbits) {
-  if (nbits < 1 || nbits > 8) return 0;
+  if (nbits < 1 || nbits > kMaxNbits) return 0;
   const StreamLayout L = stream_layout(n, 1u << nbits);
   return L.payload_off + (n * (uint64_t)nbits + 7) / 8 + 16 * L.nchunks;
 }
@@ -104,13 +104,14 @@ int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbit
 int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                     uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
                     uint32_t options, lc_cuda_stream_t cs) {
-  if (options & ~(uint32_t)LC_OPT_NO_DEVICE_WAIT) return LC_ERR_ARG;
+  if (options & ~(uint32_t)(LC_OPT_NO_DEVICE_WAIT | LC_OPT_FIXED_WIDTH)) return LC_ERR_ARG;
   if (tracked_out) {
     const int rc = check_tracked_out(cur, n, tracked_out);
     if (rc != LC_OK) return rc;
   }
   EncodeOptions opt;
   opt.two_pass_scan = (options & LC_OPT_NO_DEVICE_WAIT) != 0;
+  opt.fixed_width = (options & LC_OPT_FIXED_WIDTH) != 0;
   return compress_impl(base, cur, n, nbits, stream, stream_capacity, tracked_out, workspace, workspace_bytes, opt, cs);
 }
 
@@ -127,7 +128,7 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
                       uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs,
                       float* kernel_ms) {
   if (!kernel_ms) return LC_ERR_ARG;
-  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (nbits < 1 || nbits > kMaxNbits || n >= (1ull << 32)) return LC_ERR_ARG;
   if (!stream || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
   if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
     return LC_ERR_ARG;
@@ -141,7 +142,7 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
   ok = ok && cudaEventRecord(ev[0], cs) == cudaSuccess;
   ok = ok && launch_stats(base, cur, n, c.ctl, c.plane, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[1], cs) == cudaSuccess;
-  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, cs) == cudaSuccess;
+  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, false, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[2], cs) == cudaSuccess;
   ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[3], cs) == cudaSuccess;
@@ -181,7 +182,7 @@ int lc_recover(const float* base, const void* const* streams, const uint64_t* st
 int lc_compress_async(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                       uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs_state,
                       lc_cuda_stream_t cs_side, lc_cuda_event_t state_read) {
-  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (nbits < 1 || nbits > kMaxNbits || n >= (1ull << 32)) return LC_ERR_ARG;
   if (!stream || !workspace || !state_read || cs_state == cs_side || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
   if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(workspace, 256))
     return LC_ERR_ARG;
@@ -194,7 +195,7 @@ int lc_compress_async(const float* base, const float* cur, uint64_t n, int nbits
   if (cudaEventRecord(state_read, cs_state) != cudaSuccess) return LC_ERR_CUDA;
   // beside whatever cs_state does next: table and encode, which work on the bucket statistics and the key plane
   if (cudaStreamWaitEvent(cs_side, state_read, 0) != cudaSuccess) return LC_ERR_CUDA;
-  if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), /*wide_ok=*/false, cs_side) != cudaSuccess)
+  if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), /*wide_ok=*/false, false, cs_side) != cudaSuccess)
     return LC_ERR_CUDA;
   if (launch_encode(c.ctl, c.tiles, c.plane, nullptr, nullptr, n, static_cast<uint8_t*>(stream), nullptr,
                     EncodeOptions(), cs_side) != cudaSuccess)
@@ -205,7 +206,7 @@ int lc_compress_async(const float* base, const float* cur, uint64_t n, int nbits
 int lc_merge(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k, uint64_t n,
              int nbits, void* stream, uint64_t stream_capacity, float* scratch, void* workspace,
              uint64_t workspace_bytes, lc_cuda_stream_t cs) {
-  if (nbits < 1 || nbits > 8) return LC_ERR_ARG;
+  if (nbits < 1 || nbits > kMaxNbits) return LC_ERR_ARG;
   if (!stream || !aligned(stream, 16) || (n > 0 && (!scratch || !aligned(scratch, 16) || scratch == base)))
     return LC_ERR_ARG;
   if (workspace_bytes < workspace_layout(n).total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
@@ -231,6 +232,7 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
   };
   memset(info, 0, sizeof *info);
   info->nbits = h[6];
+  info->fixed_width = h[7] & 1u;
   info->n = le(8, 8);
   info->nsym = (uint32_t)le(16, 4);
   info->max_len = (uint32_t)le(20, 4);
@@ -238,7 +240,7 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
   info->payload_bits = le(40, 8);
   info->total_bytes = le(48, 8);
   info->payload_offset = le(56, 8);
-  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 &&
+  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 && h[7] <= 1 &&
                  le(24, 4) == kChunkElems && le(28, 2) == kLanes && le(30, 2) == kGroup &&
                  le(36, 4) == kPayloadAlign)
                     ? 1
@@ -258,7 +260,7 @@ int lc_last_status(const void* workspace, lc_cuda_stream_t cs) {
 // ---- host-buffer variants ------------------------------------------------------------------------
 
 uint64_t lc_host_arena_bytes(uint64_t n, int nbits, int k) {
-  if (nbits < 1 || nbits > 8 || k < 1 || k > LC_MAX_CHAIN) return 0;
+  if (nbits < 1 || nbits > kMaxNbits || k < 1 || k > LC_MAX_CHAIN) return 0;
   const uint64_t vec = align_up(4 * n, 256);
   const uint64_t str = align_up(lc_stream_bound(n, nbits), 256);
   const uint64_t compress = 2 * vec + str;
@@ -269,7 +271,7 @@ uint64_t lc_host_arena_bytes(uint64_t n, int nbits, int k) {
 int lc_compress_host(const float* base_host, const float* cur_host, uint64_t n, int nbits, void* stream_host,
                      uint64_t stream_capacity, uint64_t* stream_bytes_out, void* arena, uint64_t arena_bytes,
                      lc_cuda_stream_t cs) {
-  if (nbits < 1 || nbits > 8 || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (nbits < 1 || nbits > kMaxNbits || n >= (1ull << 32)) return LC_ERR_ARG;
   if (!stream_host || !stream_bytes_out || !arena || !aligned(arena, 256) || (n > 0 && (!base_host || !cur_host)))
     return LC_ERR_ARG;
   const uint64_t bound = lc_stream_bound(n, nbits);

@@ -17,6 +17,8 @@ constexpr uint32_t kHeaderBytes = 64;
 constexpr uint32_t kTableEntryBytes = 16;
 constexpr uint32_t kPayloadAlign = 16;
 constexpr uint32_t kKeys = 512;  // 256*sign + exponent field
+constexpr int kMaxNbits = 9;     // 9 keeps every occupied bucket (at most 508 of them, plus the zero symbol)
+constexpr uint32_t kMaxSymbols = 512;
 
 __host__ __device__ inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
@@ -115,6 +117,7 @@ struct EncodeOptions {
   bool two_pass_scan = false;     // offsets from a sizes pass and a one-CTA scan: no CTA ever waits for another
   uint32_t spin_limit = 1u << 20; // polls of the look-back before it gives up with LC_ERR_TIMEOUT
   uint32_t ticket_bias = 0;       // added to every tile ticket (test aid: with 1, tile 0 is never coded)
+  bool fixed_width = false;       // fixed-width codes (format section 1.5) instead of the Huffman code
 };
 
 // ---- launchers (each defined next to its kernel) ---------------------------------------------------
@@ -122,7 +125,9 @@ cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Contro
                          cudaStream_t cs);
 // wide_ok: false if the encode pass will not be able to read base and cur (the table pass then rejects a vector
 // with an exponent field >= 128 with LC_ERR_RANGE)
-cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, cudaStream_t cs);
+// fixed: fixed-width codes (format section 1.5) instead of the Huffman code
+cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, bool fixed,
+                         cudaStream_t cs);
 // tracked_out: nullptr, or where to write base + quantized delta (may be base itself)
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
                           const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, const EncodeOptions& opt,

@@ -60,7 +60,7 @@ static_assert((1 << kL1Bits) * kL1Rep * 8 == kTableBytes, "table sizes");
 struct alignas(16) StreamState {
   uint2* l1;  // [(1 << kL1Bits) * kL1Rep] {bit pattern of rep, code length}; length kLongCode = not resolved here
   uint2* sub; // 8 KB of sub-tables of (1 << sub_bits) entries: {rep, length} or length kLongCode = longer code
-  uint32_t sorted_rep[256];           // representatives in canonical (len, id) order
+  uint32_t sorted_rep[kMaxSymbols];   // representatives in canonical (len, id) order
   unsigned long long first_code[64];  // first canonical code of each length
   unsigned long long last_aligned[64]; // largest left-aligned 64-bit window whose code has at most this length
   uint32_t len_count[64];             // codes of each length
@@ -69,12 +69,13 @@ struct alignas(16) StreamState {
   unsigned long long n, payload_bits, total_bytes, payload_off, payload_size;
   unsigned long long chunk_index_off, lane_index_off;
   uint32_t nsym, max_len, nchunks, only_rep;
+  uint32_t fixed;  // fixed-width codes (format section 1.5): every symbol is coded, used or not
   // validation accumulators
   unsigned long long kraft, count_sum, bit_sum;
   uint32_t seen_max, nused, nsub;
   uint32_t sub_bits;  // depth of the sub-tables, kSubBitsMin..kSubBitsMax: as many as 8 KB hold at that depth
   uint8_t sub_of_prefix[1 << kL1Bits], prefix_of_sub[1 << kL1Bits];
-  uint8_t sym_len[256];   // code length by symbol id
+  uint8_t sym_len[kMaxSymbols];  // code length by symbol id
   uint32_t miss_count[2];  // first-level prefixes without a short code, per warp of 32 prefixes
   alignas(16) uint8_t hdr[kHeaderBytes];  // the stream header, staged
 };
@@ -118,7 +119,8 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
       S.total_bytes = load_le(h + 48, 8);
       S.payload_off = load_le(h + 56, 8);
       const bool magic = h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1';
-      if (!magic || load_le(h + 4, 2) != 1 || nbits < 1 || nbits > 8 || h[7] != 0) err = LC_ERR_FORMAT;
+      S.fixed = h[7] & 1u;
+      if (!magic || load_le(h + 4, 2) != 1 || nbits < 1 || nbits > (uint32_t)kMaxNbits || h[7] > 1) err = LC_ERR_FORMAT;
       else if (S.nsym < 1 || S.nsym > (1u << nbits) || S.max_len > 63) err = LC_ERR_FORMAT;
       else if (load_le(h + 24, 4) != kChunkElems || load_le(h + 28, 2) != kLanes ||
                load_le(h + 30, 2) != kGroup || load_le(h + 36, 4) != kPayloadAlign) err = LC_ERR_FORMAT;
@@ -144,24 +146,27 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   __syncthreads();
   if (*s_err) return *s_err;
 
-  // ---- table entries: one thread per symbol
+  // ---- table entries: a thread per symbol (up to 509 symbols, CTAs of 256 threads and more)
   const uint32_t nsym = S.nsym;
-  uint32_t my_len = 0, my_rep = 0;
-  unsigned long long my_count = 0;
+  const bool fixed = S.fixed != 0;
+  uint32_t fixed_width = 0;
+  while ((1u << fixed_width) < nsym) fixed_width += 1;
   bool entry_bad = false;
-  if (tid < (int)nsym) {
-    const uint4 e = __ldg(reinterpret_cast<const uint4*>(s + kHeaderBytes) + tid);  // key:16 len:8 pad:8 | rep | count
-    my_len = (e.x >> 16) & 255u;
-    my_rep = e.y;
-    my_count = ((unsigned long long)e.w << 32) | e.z;
-    entry_bad = (e.x >> 24) != 0 || my_len > 63 || (my_count == 0 && my_len != 0);
-    S.sym_len[tid] = (uint8_t)my_len;
+  for (uint32_t sym = tid; sym < nsym; sym += nthreads) {
+    const uint4 e = __ldg(reinterpret_cast<const uint4*>(s + kHeaderBytes) + sym);  // key:16 len:8 pad:8 | rep | count
+    const uint32_t my_len = (e.x >> 16) & 255u, my_rep = e.y;
+    const unsigned long long my_count = ((unsigned long long)e.w << 32) | e.z;
+    entry_bad |= (e.x >> 24) != 0 || my_len > 63;
+    entry_bad |= fixed ? (my_len != fixed_width) : (my_count == 0 && my_len != 0);
+    S.sym_len[sym] = (uint8_t)my_len;
     if (my_count != 0) {
       atomicAdd(&S.count_sum, my_count);
       atomicAdd(&S.bit_sum, my_count * my_len);
-      atomicAdd(&S.nused, 1u);
       atomicMax(&S.seen_max, my_len);
-      S.only_rep = my_rep;  // meaningful only when a single symbol is used
+    }
+    if (fixed ? (fixed_width > 0 || sym == 0) : (my_count != 0)) {  // the symbols that have a code
+      atomicAdd(&S.nused, 1u);
+      if (fixed ? sym == 0 : true) S.only_rep = my_rep;  // meaningful only when a single symbol is coded
       if (my_len > 0 && my_len <= 63) {
         atomicAdd(&S.kraft, 1ull << (63 - my_len));
         atomicAdd(&S.len_count[my_len], 1u);
@@ -171,11 +176,18 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   if (__syncthreads_or(entry_bad)) return LC_ERR_FORMAT;
   if (tid == 0) {
     int err = 0;
-    if (S.count_sum != S.n || S.bit_sum != S.payload_bits || S.seen_max != S.max_len) err = LC_ERR_FORMAT;
-    if (S.nused >= 2) {
-      if (S.kraft != (1ull << 63)) err = LC_ERR_FORMAT;
-    } else if (S.max_len != 0) {
-      err = LC_ERR_FORMAT;
+    if (S.count_sum != S.n || S.bit_sum != S.payload_bits) err = LC_ERR_FORMAT;
+    if (S.fixed) {
+      uint32_t width = 0;
+      while ((1u << width) < S.nsym) width += 1;
+      if (S.max_len != width) err = LC_ERR_FORMAT;  // every entry's length was compared with the width above
+    } else {
+      if (S.seen_max != S.max_len) err = LC_ERR_FORMAT;
+      if (S.nused >= 2) {
+        if (S.kraft != (1ull << 63)) err = LC_ERR_FORMAT;
+      } else if (S.max_len != 0) {
+        err = LC_ERR_FORMAT;
+      }
     }
     // canonical first codes per length
     unsigned long long code = 0;
@@ -197,11 +209,15 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   }
   __syncthreads();
   if (*s_err) return *s_err;
-  if (S.nused >= 2 && tid < (int)nsym && my_count != 0) {
-    // rank among the symbols of the same length with smaller id (zero-count symbols have length 0)
-    uint32_t r = 0;
-    for (int j = 0; j < tid; ++j) r += (S.sym_len[j] == my_len) ? 1u : 0u;
-    S.sorted_rep[S.len_offset[my_len] + r] = my_rep;
+  if (S.nused >= 2) {
+    for (uint32_t sym = tid; sym < nsym; sym += nthreads) {
+      const uint32_t my_len = S.sym_len[sym];
+      if (my_len == 0) continue;  // a symbol without a code (unused, in a Huffman-coded stream)
+      // rank among the symbols of the same length with smaller id
+      uint32_t r = 0;
+      for (uint32_t j = 0; j < sym; ++j) r += (S.sym_len[j] == my_len) ? 1u : 0u;
+      S.sorted_rep[S.len_offset[my_len] + r] = __ldg(reinterpret_cast<const uint32_t*>(s + kHeaderBytes + 16 * sym + 4));
+    }
   }
   if (S.nused < 2 && tid == 0) S.sorted_rep[0] = S.only_rep;
   __syncthreads();

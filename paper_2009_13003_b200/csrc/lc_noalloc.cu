@@ -41,7 +41,7 @@ int scratch_for_current_device(void** out) {
 
 extern "C" int lc_compress_noalloc(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                                    uint64_t stream_capacity, lc_cuda_stream_t cs) {
-  if (nbits < 1 || nbits > 8) return LC_ERR_ARG;
+  if (nbits < 1 || nbits > kMaxNbits) return LC_ERR_ARG;
   if (n > kNoAllocMaxN) return LC_ERR_CAPACITY;  // beyond the built-in scratch: use lc_compress
   if (!stream || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
   if ((reinterpret_cast<uintptr_t>(base) | reinterpret_cast<uintptr_t>(cur) | reinterpret_cast<uintptr_t>(stream)) & 15)
@@ -61,7 +61,7 @@ extern "C" int lc_compress_noalloc(const float* base, const float* cur, uint64_t
   // the array keeps what the previous call left: counters, bins and tile descriptors must start at zero
   if (cudaMemsetAsync(w, 0, W.plane_off, cs) != cudaSuccess) return LC_ERR_CUDA;
   if (launch_stats(base, cur, n, ctl, plane, cs) != cudaSuccess) return LC_ERR_CUDA;
-  if (launch_table(ctl, n, nbits, static_cast<uint8_t*>(stream), true, cs) != cudaSuccess) return LC_ERR_CUDA;
+  if (launch_table(ctl, n, nbits, static_cast<uint8_t*>(stream), true, false, cs) != cudaSuccess) return LC_ERR_CUDA;
   if (launch_encode(ctl, tiles, plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(), cs) != cudaSuccess)
     return LC_ERR_CUDA;
   int32_t status = 0;

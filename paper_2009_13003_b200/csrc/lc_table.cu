@@ -13,14 +13,15 @@ namespace lc {
 namespace {
 
 constexpr int kTableThreads = 512;
-constexpr int kMaxSym = 256;
+constexpr int kMaxSym = kMaxSymbols;
 
 __device__ __forceinline__ void store_le(uint8_t* p, uint64_t v, int bytes) {
   for (int b = 0; b < bytes; ++b) p[b] = (uint8_t)(v >> (8 * b));
 }
 
 __global__ void __launch_bounds__(kTableThreads)
-table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restrict__ stream, int wide_ok) {
+table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restrict__ stream, int wide_ok,
+             int fixed) {
   __shared__ uint32_t warp_cand[16];
   __shared__ uint16_t sym_of_key[kKeys];
   __shared__ unsigned long long sym_count[kMaxSym];
@@ -131,11 +132,24 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     used = my_count != 0;
   }
   const uint32_t used_ballot = __ballot_sync(0xffffffffu, used);
-  if (lane == 0 && warp < 8) warp_cand[warp] = __popc(used_ballot);
+  if (lane == 0) warp_cand[warp] = __popc(used_ballot);
   __syncthreads();
   uint32_t nused = 0;
-  for (int w = 0; w < 8; ++w) nused += warp_cand[w];
-  if (used) {
+  for (int w = 0; w < 16; ++w) nused += warp_cand[w];
+  if (fixed) {
+    // fixed-width codes (format section 1.5): every symbol, used or not, takes ceil(log2 nsym) bits; its code is its id
+    uint32_t width = 0;
+    while ((1u << width) < nsym) width += 1;
+    if (tid < (int)nsym) {
+      sym_len[tid] = width;
+      sym_code[tid] = (unsigned long long)tid;
+    }
+    if (tid == 0) {
+      s_maxlen = width;
+      s_payload_bits = n * width;
+    }
+  }
+  if (used && !fixed) {
     uint32_t r = 0;
     for (uint32_t j = 0; j < nsym; ++j) {
       const unsigned long long cj = sym_count[j];
@@ -145,7 +159,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     leaf_sym[r] = (uint16_t)tid;
   }
   __syncthreads();
-  if (tid == 0 && nused >= 2) {
+  if (tid == 0 && nused >= 2 && !fixed) {
     uint32_t front_a = 0, front_b = nused, next = nused;
     for (uint32_t merge = 0; merge + 1 < nused; ++merge) {
       uint32_t pick[2];
@@ -176,7 +190,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   __syncthreads();
 
   // ---- canonical codes: used symbols sorted by (len, id) -------------------------------------------
-  if (used && nused >= 2) {
+  if (used && nused >= 2 && !fixed) {
     const uint32_t my_len = sym_len[tid];
     uint32_t r = 0;
     for (uint32_t j = 0; j < nsym; ++j) {
@@ -186,7 +200,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     canon_order[r] = (uint16_t)tid;
   }
   __syncthreads();
-  if (tid == 0 && nused >= 2) {
+  if (tid == 0 && nused >= 2 && !fixed) {
     unsigned long long code = 0;
     uint32_t prev_len = 0;
     for (uint32_t r = 0; r < nused; ++r) {
@@ -226,7 +240,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
     store_le(h + 4, 1, 2);
     h[6] = (uint8_t)nbits;
-    h[7] = 0;
+    h[7] = (uint8_t)(fixed ? 1 : 0);
     store_le(h + 8, n, 8);
     store_le(h + 16, nsym, 4);
     store_le(h + 20, s_maxlen, 4);
@@ -249,8 +263,9 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
 
 }  // namespace
 
-cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, cudaStream_t cs) {
-  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0);
+cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, bool fixed,
+                         cudaStream_t cs) {
+  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0, fixed ? 1 : 0);
   return cudaGetLastError();
 }
 

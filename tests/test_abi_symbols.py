@@ -27,13 +27,13 @@ def test_host_side_size_functions_match_the_format_text(oracle):
     from paper_2009_13003_b200 import binding
 
     for n in (0, 1, 10, 4096, 4097, 61_706, 11_689_512, 1_315_575_808):
-        for nbits in (1, 2, 5, 8):
+        for nbits in (1, 2, 5, 8, 9):
             nchunks = (n + 4095) // 4096
             head = (64 + 16 * 2 ** nbits + 8 * (nchunks + 1) + 64 * nchunks + 15) // 16 * 16
             want = head + (n * nbits + 7) // 8 + 16 * nchunks
             assert binding.stream_bound(n, nbits) == want == oracle.stream_bound(n, nbits)
         assert n <= binding.workspace_bytes(n) <= 1.01 * n + 65536
-    assert binding.stream_bound(10, 0) == 0 and binding.stream_bound(10, 9) == 0
+    assert binding.stream_bound(10, 0) == 0 and binding.stream_bound(10, 10) == 0
 
 
 def test_host_argument_checks_need_no_device():
@@ -49,11 +49,11 @@ def test_host_argument_checks_need_no_device():
     assert upd(None) == binding.ERR_ARG
     assert upd(cur) == binding.ERR_ARG
     assert upd(0x50004) == binding.ERR_ARG
-    assert upd(0x50000, nbits=9) == binding.ERR_ARG
+    assert upd(0x50000, nbits=10) == binding.ERR_ARG
     assert L.lc_compress_update(base, cur, 16, 4, stream, 8, 0x50000, ws, 1 << 20, None) == binding.ERR_CAPACITY
     assert L.lc_strerror(binding.ERR_FORMAT) == b"malformed stream"
     # lc_compress_opt: unknown option bits are refused before anything else happens
-    assert L.lc_compress_opt(base, cur, 16, 4, stream, 1 << 20, None, ws, 1 << 20, 2, None) == binding.ERR_ARG
+    assert L.lc_compress_opt(base, cur, 16, 4, stream, 1 << 20, None, ws, 1 << 20, 4, None) == binding.ERR_ARG
     assert L.lc_compress_opt(base, cur, 16, 4, stream, 1 << 20, cur, ws, 1 << 20, 1, None) == binding.ERR_ARG
 
 

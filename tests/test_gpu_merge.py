@@ -82,7 +82,7 @@ def test_merge_reports_a_rejected_stream_and_bad_arguments(lc):
     sizes = (C.c_uint64 * 2)(*[s.numel() for s in streams])
     args = lambda nbits=4, scr=scratch.data_ptr(), cap=out.numel(): (u0.data_ptr(), ptrs, sizes, 2, n, nbits, out.data_ptr(), cap,
                                                                     scr, ws.data_ptr(), ws.numel(), None)
-    assert L.lc_merge(*args(nbits=9)) == lc.ERR_ARG
+    assert L.lc_merge(*args(nbits=10)) == lc.ERR_ARG
     assert L.lc_merge(*args(scr=None)) == lc.ERR_ARG
     assert L.lc_merge(*args(scr=u0.data_ptr())) == lc.ERR_ARG
     assert L.lc_merge(*args(cap=100)) == lc.ERR_CAPACITY

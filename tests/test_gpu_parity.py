@@ -381,7 +381,7 @@ def test_argument_errors(lc):
     L = lc.lib()
     cs = None
     assert L.lc_compress(base.data_ptr(), cur.data_ptr(), 5000, 0, st.data_ptr(), st.numel(), ws.data_ptr(), ws.numel(), cs) == lc.ERR_ARG
-    assert L.lc_compress(base.data_ptr(), cur.data_ptr(), 5000, 9, st.data_ptr(), st.numel(), ws.data_ptr(), ws.numel(), cs) == lc.ERR_ARG
+    assert L.lc_compress(base.data_ptr(), cur.data_ptr(), 5000, 10, st.data_ptr(), st.numel(), ws.data_ptr(), ws.numel(), cs) == lc.ERR_ARG
     assert L.lc_compress(None, cur.data_ptr(), 5000, 4, st.data_ptr(), st.numel(), ws.data_ptr(), ws.numel(), cs) == lc.ERR_ARG
     assert L.lc_compress(base.data_ptr() + 4, cur.data_ptr(), 4999, 4, st.data_ptr(), st.numel(), ws.data_ptr(), ws.numel(), cs) == lc.ERR_ARG
     assert L.lc_compress(base.data_ptr(), cur.data_ptr(), 5000, 4, st.data_ptr(), st.numel() - 1, ws.data_ptr(), ws.numel(), cs) == lc.ERR_CAPACITY
@@ -425,7 +425,7 @@ def test_corrupted_streams_are_rejected_not_faulting(lc, oracle):
     assert status_of(good) == 0
     assert status_of(mutated(0, ord("X"))) == lc.ERR_FORMAT       # magic
     assert status_of(mutated(4, 2)) == lc.ERR_FORMAT              # version
-    assert status_of(mutated(6, 9)) == lc.ERR_FORMAT              # nbits
+    assert status_of(mutated(6, 10)) == lc.ERR_FORMAT             # nbits
     assert status_of(mutated(16, 200)) == lc.ERR_FORMAT           # nsym
     assert status_of(mutated(24, 1)) == lc.ERR_FORMAT             # chunk_elems
     assert status_of(mutated(64 + 16 + 2, 1)) == lc.ERR_FORMAT    # a code length: Kraft / bit count

@@ -56,6 +56,8 @@ MUTATIONS = [
     ("threaded statistics: minimum not merged", "if (b.vmin < m.vmin) m.vmin = b.vmin;", "if (b.vmin > m.vmin) m.vmin = b.vmin;"),
     ("threaded recovery: chunk range off by one", "const uint64_t lo = c * kChunkElems, hi = std::min(n, lo + kChunkElems);\n        if (parsed[j].table.max_len == 0)",
      "const uint64_t lo = c * kChunkElems, hi = std::min(n, lo + kChunkElems - 1);\n        if (parsed[j].table.max_len == 0)"),
+    ("fixed width one bit short", "while ((1 << width) < t->nsym) width += 1;", "while ((2 << width) < t->nsym) width += 1;"),
+    ("fixed-width code is not the symbol id", "t->code[j] = static_cast<uint64_t>(j);", "t->code[j] = static_cast<uint64_t>(t->nsym - 1 - j);"),
     ("size model uses floor log", "while ((1ull << width) < k) width += 1;", "while ((2ull << width) <= k) width += 1;"),
 ]
 
@@ -84,12 +86,21 @@ class _Oracle:
         L.lco_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp]
         L.lco_midrange.argtypes = [C.c_float, C.c_float]
         L.lco_midrange.restype = C.c_float
+        L.lco_compress_mode.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64)]
         L.lco_apply_quantized.argtypes = [vp, vp, u64, i32, vp]
         L.lco_compress_chunks.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
         L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_mt.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), i32]
         L.lco_recover_mt.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, i32]
         self.L = L
+
+    def compress_fixed(self, base, cur, nbits):
+        cap = int(self.L.lco_stream_bound(base.size, nbits))
+        buf = np.zeros(cap + 64, np.uint8)
+        out = C.c_uint64(0)
+        assert self.L.lco_compress_mode(base.ctypes.data, cur.ctypes.data, base.size, nbits, 1, buf.ctypes.data, cap,
+                                        C.byref(out)) == 0
+        return buf[: out.value].copy()
 
     def apply_quantized(self, base, cur, nbits):
         out = np.zeros(base.size, np.float32)
@@ -245,6 +256,25 @@ def _pins_hold(o):
             return False
         m = o.merge(base, [s, s], 3)
         if not np.array_equal(o.recover(base, [m]).view(np.uint32), o.apply_quantized(base, out, 3).view(np.uint32)):
+            return False
+        # fixed-width codes on the paper's example: 10 elements, 5 buckets, 3-bit indices -> 30 payload bits, first
+        # payload word = the ids of the four elements of lane 0, then lane 1, ... most significant bit first
+        g = load_golden("ten_elements_nbits2.txt")
+        zb = np.zeros(10, np.float32)
+        sf = o.compress_fixed(zb, g["cur"], 9)
+        if int(np.frombuffer(sf[40:48].tobytes(), "<u8")[0]) != 30 or sf[20] != 3:
+            return False
+        if o.recover(zb, [sf]).view(np.uint32).tolist() != o.apply_quantized(zb, g["cur"], 9).view(np.uint32).tolist():
+            return False
+        # the Huffman stream of the same vector tells the symbol of every element; the fixed code of symbol j is j
+        pof = int(np.frombuffer(sf[56:64].tobytes(), "<u8")[0])
+        word0 = int(np.frombuffer(sf[pof:pof + 4].tobytes(), "<u4")[0])
+        cur10 = g["cur"]
+        keys = [(int(v.view(np.uint32)) >> 31) * 256 + ((int(v.view(np.uint32)) >> 23) & 255) for v in cur10]
+        order = sorted(set(keys), key=lambda k: (-(k % 256), k // 256))
+        ids = [order.index(k) + 1 for k in keys]
+        want_bits = "".join(format(i, "03b") for i in ids).ljust(32, "0")
+        if word0 != int(want_bits, 2):
             return False
         # the threaded timing mode writes the same bytes and states
         if o.compress_mt(base, cur, 3, 3).tobytes() != s.tobytes():

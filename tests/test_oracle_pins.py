@@ -414,7 +414,8 @@ def test_reader_rejects_corruption(oracle):
 
     expect(setb(0, ord("X")), oracle.ERR_FORMAT)     # magic
     expect(setb(4, 2), oracle.ERR_FORMAT)            # version
-    expect(setb(6, 9), oracle.ERR_FORMAT)            # nbits
+    expect(setb(6, 10), oracle.ERR_FORMAT)           # nbits
+    expect(setb(7, 2), oracle.ERR_FORMAT)            # flags
     expect(setb(16, 200), oracle.ERR_FORMAT)         # nsym > 2^nbits
     expect(setb(24, 1), oracle.ERR_FORMAT)           # chunk_elems
     expect(setb(64 + 16 + 2, 1), oracle.ERR_FORMAT)  # a code length changed: Kraft / payload_bits
@@ -545,3 +546,114 @@ def test_merge_is_compress_of_the_recovered_state(oracle):
         assert np.array_equal(back.view(np.uint32), (u0 + t4["rep"][sym]).view(np.uint32))
     with pytest.raises(oracle.OracleError):
         oracle.merge(u0[:-1], streams[:1], 4)  # element count mismatch
+
+
+# ---------------------------------------------------------------- fixed-width codes and nbits = 9 (Section 4.3's stages)
+
+
+def _parse(s):
+    nsym = int(np.frombuffer(s[16:20].tobytes(), "<u4")[0])
+    n = int(np.frombuffer(s[8:16].tobytes(), "<u8")[0])
+    nchunks = (n + 4095) // 4096
+    ci = 64 + 16 * nsym
+    li = ci + 8 * (nchunks + 1)
+    po = int(np.frombuffer(s[56:64].tobytes(), "<u8")[0])
+    tab = np.frombuffer(s[64:ci].tobytes(), dtype=[("key", "<u2"), ("len", "u1"), ("pad", "u1"), ("rep", "<u4"), ("count", "<u8")])
+    return dict(n=n, nsym=nsym, nchunks=nchunks, tab=tab, chunk_off=np.frombuffer(s[ci:li].tobytes(), "<u8"),
+                lane_bits=np.frombuffer(s[li:li + 64 * nchunks].tobytes(), "<u2").reshape(nchunks, 32), po=po,
+                payload_bits=int(np.frombuffer(s[40:48].tobytes(), "<u8")[0]), max_len=int(s[20]), flags=int(s[7]),
+                nbits=int(s[6]))
+
+
+def test_paper_example_as_a_fixed_width_stream(oracle):
+    # Section 3.1.1's worked example: 10 elements in 5 buckets, every bucket kept (no promotion: nbits 9), fixed
+    # 3-bit indices: 10 * 3 bits of payload, and with the 5 representatives of 32 bits each 190 bits, rate 1.68.
+    g = load_golden("ten_elements_nbits2.txt")
+    base = np.zeros(10, np.float32)
+    s = oracle.compress(base, g["cur"], 9, fixed=True)
+    p = _parse(s)
+    assert p["nbits"] == 9 and p["flags"] == 1
+    assert p["nsym"] == 6 and p["max_len"] == 3 and p["payload_bits"] == 30  # 5 buckets + the zero symbol: 3 bits
+    assert p["payload_bits"] + 32 * 5 == oracle.model_bits(10, 5, 32) == 190
+    assert p["tab"]["len"].tolist() == [3] * 6 and int(p["tab"]["count"][0]) == 0
+    # nothing is dropped: every element comes back as its bucket's representative, here the element itself or
+    # the midrange of its bucket
+    out = oracle.recover(base, [s])
+    t = oracle.table(base, g["cur"], 9, fixed=True)
+    sym = oracle.symbols(base, g["cur"], 9)
+    assert np.all(sym > 0)
+    assert np.array_equal(out.view(np.uint32), t["rep"][sym].view(np.uint32))
+    # with 2-bit promotion the same vector takes 2 bits per index
+    s2 = oracle.compress(base, g["cur"], 2, fixed=True)
+    assert _parse(s2)["payload_bits"] == 20 and _parse(s2)["max_len"] == 2
+
+
+def test_fixed_width_payload_by_independent_bit_writer(oracle):
+    rng = np.random.default_rng(91)
+    n = 4096 + 777
+    base, cur = _random_case(rng, n)
+    for nbits in (1, 3, 9):
+        s = oracle.compress(base, cur, nbits, fixed=True)
+        p = _parse(s)
+        sym = oracle.symbols(base, cur, nbits)
+        width = max(0, int(p["nsym"] - 1).bit_length())
+        assert p["max_len"] == width and p["payload_bits"] == n * width
+        assert np.array_equal(oracle.decode_symbols(s, n), sym)
+        for c in range(p["nchunks"]):
+            bits = ""
+            for lane in range(32):
+                for j in range(32):
+                    for e in range(4):
+                        i = 4096 * c + 128 * j + 4 * lane + e
+                        if i < n and width:
+                            bits += format(int(sym[i]), "0%db" % width)
+            nbytes = ((len(bits) + 7) // 8 + 15) // 16 * 16
+            bits = bits.ljust(nbytes * 8, "0")
+            words = np.array([int(bits[w:w + 32], 2) for w in range(0, len(bits), 32)], "<u4")
+            lo = p["po"] + int(p["chunk_off"][c])
+            assert s[lo: p["po"] + int(p["chunk_off"][c + 1])].tobytes() == words.tobytes()
+        # same symbols and representatives as the Huffman-coded stream: the recovered state is the same
+        if nbits <= 8:
+            h = oracle.compress(base, cur, nbits)
+            assert np.array_equal(oracle.recover(base, [s]).view(np.uint32), oracle.recover(base, [h]).view(np.uint32))
+            assert s.size >= h.size - 16 * p["nchunks"]  # Huffman never needs more payload bits than the fixed code
+
+
+def test_nine_bit_promotion_keeps_every_bucket(oracle):
+    # magnitudes over 150 binades, both signs: about 300 occupied buckets, so symbol ids go beyond one byte
+    rng = np.random.default_rng(92)
+    n = 60000
+    cur = (np.exp2(rng.uniform(-100, 50, n)) * rng.choice([-1.0, 1.0], n)).astype(np.float32)
+    cur[:100] = 0.0
+    base = np.zeros(n, np.float32)
+    count, _, _ = oracle.bins(base, cur)
+    occupied = int(((count > 0) & (np.arange(512) % 256 >= 1) & (np.arange(512) % 256 <= 254)).sum())
+    assert occupied > 255
+    for fixed in (False, True):
+        s = oracle.compress(base, cur, 9, fixed=fixed)
+        p = _parse(s)
+        assert p["nsym"] == occupied + 1
+        sym = oracle.decode_symbols(s, n)
+        assert int(sym.max()) == occupied and np.array_equal(sym, oracle.symbols(base, cur, 9))
+        out = oracle.recover(base, [s])
+        d = cur
+        assert np.all(out[:100] == 0)
+        nz = d != 0
+        e = np.floor(np.log2(np.abs(d[nz])))
+        assert np.all(np.abs(out[nz].astype(np.float64) - d[nz]) < 2.0 ** (e - 1) + 1e-300)  # half a binade at most
+    assert oracle.compress(base, cur, 9, fixed=True).tobytes() == oracle.compress(base, cur, 9, fixed=True, threads=3).tobytes()
+
+
+def test_reader_checks_fixed_width_streams(oracle):
+    rng = np.random.default_rng(93)
+    base, cur = _random_case(rng, 5000)
+    good = oracle.compress(base, cur, 3, fixed=True)
+    assert oracle.recover(base, [good]).size == 5000
+    bad = good.copy()
+    bad[64 + 2] = 2  # one length changed
+    huff = oracle.compress(base, cur, 3)
+    huff[7] = 1      # a Huffman-coded stream that claims fixed-width codes
+    for s in (bad, huff):
+        with pytest.raises(oracle.OracleError) as e:
+            oracle.recover(base, [s])
+        assert e.value.code == oracle.ERR_FORMAT

@@ -54,5 +54,5 @@ def test_noalloc_rejects_sizes_beyond_its_scratch():
     buf = torch.empty(lc.stream_bound(n, 4), dtype=torch.uint8, device=DEV)
     rc = lc.lib().lc_compress_noalloc(x.data_ptr(), x.data_ptr(), n, 4, buf.data_ptr(), buf.numel(), None)
     assert rc == lc.ERR_CAPACITY
-    rc = lc.lib().lc_compress_noalloc(x.data_ptr(), x.data_ptr(), 16, 9, buf.data_ptr(), buf.numel(), None)
+    rc = lc.lib().lc_compress_noalloc(x.data_ptr(), x.data_ptr(), 16, 10, buf.data_ptr(), buf.numel(), None)
     assert rc == lc.ERR_ARG
