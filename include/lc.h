@@ -71,7 +71,7 @@ uint64_t lc_stream_bound(uint64_t n, int nbits);
 /* Bytes of DEVICE scratch lc_compress and lc_recover need for vectors of up to n elements: the control block
  * (status word, bucket statistics of Section 3.1.1, per-bucket code table), one descriptor per chunk for the
  * scan that places the chunks (format section 3.3), and one byte per element for the bucket keys that the
- * statistics pass hands to the encode pass. */
+ * statistics pass hands to the encode pass; for lc_recover, the decode tables of the streams of one launch. */
 uint64_t lc_workspace_bytes(uint64_t n);
 
 /*
@@ -141,7 +141,8 @@ int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, 
  * k             1..LC_MAX_CHAIN.
  * n             elements in base and out; every stream's header must say the same n.
  * out           DEVICE, n fp32, 16-byte aligned; may be the same pointer as base (in-place update).
- * workspace     as for lc_compress (only the status word is used).
+ * workspace     as for lc_compress; lc_workspace_bytes(0) is enough for any n (the status word and the decode
+ *               tables of the streams live there).
  * Malformed streams set LC_ERR_FORMAT / LC_ERR_MISMATCH in the status word; `out` is then unspecified
  * but no out-of-bounds access happens.
  */
@@ -240,7 +241,7 @@ int lc_recover_host(const float* base_host, const void* const* streams_host,
  *  - Every call on a device shares the one array, which keeps the previous call's contents (the call
  *    clears what must start at zero). Two calls that overlap on the same GPU race: do not issue them
  *    from different streams or threads at the same time.
- *  - The array (about 4.2 MB) stays resident on every GPU that loads the library, until exit.
+ *  - The array (about 4.3 MB) stays resident on every GPU that loads the library, until exit.
  */
 #define LC_NOALLOC_MAX_N 4194304ull
 int lc_compress_noalloc(const float* base, const float* cur, uint64_t n, int nbits, void* stream,

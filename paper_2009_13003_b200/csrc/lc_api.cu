@@ -159,8 +159,9 @@ int lc_recover(const float* base, const void* const* streams, const uint64_t* st
   if (!aligned(base, 16) || !aligned(out, 16) || !aligned(workspace, 256)) return LC_ERR_ARG;
   for (int j = 0; j < k; ++j)
     if (!streams[j] || !aligned(streams[j], 16)) return LC_ERR_ARG;
-  if (workspace_bytes < sizeof(Control)) return LC_ERR_CAPACITY;
+  if (workspace_bytes < workspace_layout(0).total) return LC_ERR_CAPACITY;
   Control* ctl = static_cast<Control*>(workspace);
+  void* images = static_cast<uint8_t*>(workspace) + workspace_layout(0).decode_off;
   cudaError_t e = cudaMemsetAsync(&ctl->status, 0, sizeof(int32_t), cs);
   if (e != cudaSuccess) return LC_ERR_CUDA;
   // up to four streams per launch; later launches continue in place from `out`.
@@ -173,7 +174,7 @@ int lc_recover(const float* base, const void* const* streams, const uint64_t* st
       ds.ptr[j] = static_cast<const uint8_t*>(streams[first + j]);
       ds.bytes[j] = stream_bytes[first + j];
     }
-    if ((e = launch_decode(src, ds, kk, n, out, &ctl->status, cs)) != cudaSuccess) return LC_ERR_CUDA;
+    if ((e = launch_decode(src, ds, kk, n, out, &ctl->status, images, cs)) != cudaSuccess) return LC_ERR_CUDA;
     src = out;
   }
   return LC_OK;

@@ -20,7 +20,7 @@ constexpr uint32_t kKeys = 512;  // 256*sign + exponent field
 constexpr int kMaxNbits = 9;     // 9 keeps every occupied bucket (at most 508 of them, plus the zero symbol)
 constexpr uint32_t kMaxSymbols = 512;
 
-__host__ __device__ inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+__host__ __device__ constexpr inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 struct StreamLayout {
   uint64_t nchunks, table_off, chunk_index_off, lane_index_off, payload_off;
@@ -82,17 +82,24 @@ struct Control {
 };
 static_assert(sizeof(Control) % 256 == 0, "control block must keep the planes 256-byte aligned");
 
+// lc_recover keeps the decode tables of the (at most four) streams of one launch behind the control block, at an
+// offset that does not depend on n: the prepare kernel builds them there once, every CTA of the decode kernel copies
+// them into its shared memory.
+constexpr uint32_t kDecodeImageBytes = 24 * 1024;  // per stream
+constexpr uint32_t kDecodeRegionBytes = 4 * kDecodeImageBytes;
+
 struct WorkspaceLayout {
-  uint64_t control_off, tiles_off, plane_off, total;
+  uint64_t control_off, decode_off, tiles_off, plane_off, total;
   uint64_t nchunks, nunits;
 };
 
-__host__ __device__ inline WorkspaceLayout workspace_layout(uint64_t n) {
-  WorkspaceLayout W;
+__host__ __device__ constexpr inline WorkspaceLayout workspace_layout(uint64_t n) {
+  WorkspaceLayout W{};
   W.nchunks = (n + kChunkElems - 1) / kChunkElems;
   W.nunits = W.nchunks * kUnitsPerChunk;
   W.control_off = 0;
-  W.tiles_off = sizeof(Control);                                // one 8-byte descriptor per chunk
+  W.decode_off = sizeof(Control);
+  W.tiles_off = W.decode_off + kDecodeRegionBytes;              // one 8-byte descriptor per chunk
   W.plane_off = align_up(W.tiles_off + 8 * W.nchunks, 256);
   W.total = align_up(W.plane_off + W.nchunks * kChunkElems, 256);  // 1 byte per element, whole chunks
   return W;
@@ -137,7 +144,8 @@ struct DecodeStreams {
   const uint8_t* ptr[4];
   uint64_t bytes[4];
 };
+// images: kDecodeRegionBytes of device scratch for the streams' decode tables (built by a first small kernel)
 cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
-                          int32_t* status, cudaStream_t cs);
+                          int32_t* status, void* images, cudaStream_t cs);
 
 }  // namespace lc

@@ -278,6 +278,46 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
   return 0;
 }
 
+// What the prepare kernel leaves in global memory for one stream and every CTA of the decode kernel copies: the two
+// lookup tables, the stream's state, and the outcome of the validation. First-level entries that point to a sub-table
+// hold that table's offset from the start of the sub-table area there (the shared address is added by the copy).
+struct DecodeImage {
+  uint2 l1[kTableBytes / 8];
+  uint2 sub[kTableBytes / 8];
+  StreamState state;
+  int32_t err;
+  int32_t pad_[3];
+};
+static_assert(sizeof(DecodeImage) <= kDecodeImageBytes, "the workspace region holds four of these");
+static_assert(sizeof(DecodeImage) % 16 == 0 && sizeof(StreamState) % 16 == 0, "copied with 16-byte accesses");
+
+constexpr int kPrepThreads = 512;
+constexpr uint32_t kPrepSmem = kTableBytes + 2 * kTableBytes + sizeof(StreamState);
+
+// One CTA per stream: parse, validate, build the tables (in this CTA's shared memory, as the decode kernel would),
+// then write the image.
+__global__ void __launch_bounds__(kPrepThreads)
+decode_prepare_kernel(DecodeStreams streams, uint64_t n, DecodeImage* __restrict__ images) {
+  extern __shared__ __align__(16) unsigned char p_raw[];
+  unsigned char* tables = p_raw + ((kTableBytes - (smem_addr(p_raw) & (kTableBytes - 1))) & (kTableBytes - 1));
+  StreamState& S = *reinterpret_cast<StreamState*>(p_raw + kTableBytes + 2 * kTableBytes);
+  __shared__ int s_err;
+  DecodeImage& img = images[blockIdx.x];
+  const int err = prepare_stream(S, tables, streams.ptr[blockIdx.x], streams.bytes[blockIdx.x], n, &s_err);
+  if (threadIdx.x == 0) img.err = err;
+  if (err) return;
+  const uint32_t sub_addr = smem_addr(S.sub);
+  for (uint32_t k = threadIdx.x; k < kTableBytes / 8; k += kPrepThreads) {
+    uint2 e = S.l1[k];
+    if (e.y == kLongCode) e.x -= sub_addr;
+    img.l1[k] = e;
+    img.sub[k] = S.sub[k];
+  }
+  const uint4* src = reinterpret_cast<const uint4*>(&S);
+  uint4* dst = reinterpret_cast<uint4*>(&img.state);
+  for (uint32_t k = threadIdx.x; k < sizeof(StreamState) / 16; k += kPrepThreads) dst[k] = src[k];
+}
+
 // Two-level table lookup of the code at the top of `hi`: {representative, length}, length kLongCode if
 // the tables do not resolve it. `l1lane` = shared address of this lane's copy of first-level entry 0.
 // The first-level entry of a prefix that belongs to longer codes holds the shared address of the
@@ -301,25 +341,6 @@ __device__ __forceinline__ uint2 lookup_code(uint32_t hi, uint32_t l1lane, uint3
       : "=&r"(ent.x), "=&r"(ent.y)
       : "r"(hi), "r"(l1lane), "n"(32 - kL1Bits), "n"(kL1Rep * 8), "n"(kL1Bits), "r"(sub_shift), "n"(OFFSET));
   return ent;
-}
-
-// Table-free canonical decode of the code that starts at bit `bitpos` of a chunk in global memory
-// (the slow path for ragged or oversized chunks): {representative, length}.
-__device__ __noinline__ uint2 decode_any(const StreamState& S, const uint32_t* g, uint32_t nw, uint32_t bitpos,
-                                         int32_t* status) {
-  if (S.nused < 2) return make_uint2(S.only_rep, 0u);
-  auto rd = [&](uint32_t i) { return i < nw ? __ldg(g + i) : 0u; };
-  const uint32_t wi = bitpos >> 5, p = bitpos & 31;
-  const unsigned long long a = ((unsigned long long)rd(wi) << 32) | rd(wi + 1);
-  const unsigned long long b = rd(wi + 2);
-  const unsigned long long window = p ? ((a << p) | (b >> (32 - p))) : a;
-  for (uint32_t L = 1; L <= S.max_len; ++L) {
-    const unsigned long long c = window >> (64 - L);
-    if (c >= S.first_code[L] && c - S.first_code[L] < S.len_count[L])
-      return make_uint2(S.sorted_rep[S.len_offset[L] + (uint32_t)(c - S.first_code[L])], L);
-  }
-  set_status(status, LC_ERR_FORMAT);  // no code matches: damaged payload
-  return make_uint2(0u, S.max_len);
 }
 
 // Code the tables did not resolve: canonical search on a 64-bit window read from the chunk, then re-seat
@@ -458,28 +479,37 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
 }
 static_assert(kL1Rep * 8 == 128, "first-level entries of one index span 128 bytes");
 
-// The ragged last chunk, read from global memory; plain code, no warp votes.
-struct GlobalChunk {
-  const uint32_t* g[4];
-  uint32_t nw[4];
+// The vector's last, partial chunk: element by element (indices beyond n are skipped), each code with a top-up, a
+// table lookup and, if the tables do not resolve it, the canonical search. Out of line: it runs once per call, in one
+// warp, and must not weigh on the registers of the loop above. The chunk's words come from the staging areas if
+// they fit there (a single warp waiting for global memory at every code would take several times as long as all the
+// other chunks of a medium-sized vector together), else from global memory.
+struct PartialChunk {
+  Source W[4];
   uint32_t start[4];
+  uint32_t sub_shift[4];
 };
-template <int KS>
-__device__ __noinline__ void decode_chunk_global(const StreamState* S, GlobalChunk G, const float* base, float* out,
-                                                 uint64_t c, uint64_t n, uint32_t lane, int32_t* status) {
-  uint32_t pos[KS];
+template <int KS, bool STAGED>
+__device__ __noinline__ void decode_chunk_partial(const StreamState* S, PartialChunk P, uint32_t l1lane,
+                                                  const float* base, float* out, uint64_t c, uint64_t n, uint32_t lane,
+                                                  int32_t* status) {
+  LaneBits<STAGED> bits[KS];
 #pragma unroll
-  for (int s = 0; s < KS; ++s) pos[s] = G.start[s];
+  for (int s = 0; s < KS; ++s) bits[s].seek(P.W[s], P.start[s]);
+#pragma unroll 1
   for (uint32_t j = 0; j < kSteps; ++j) {
+#pragma unroll 1
     for (uint32_t e = 0; e < kGroup; ++e) {
       const uint64_t i = c * kChunkElems + 128ull * j + 4 * lane + e;
       if (i >= n) continue;
       float x = base[i];
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        const uint2 ent = decode_any(S[s], G.g[s], G.nw[s], pos[s], status);
+        bits[s].refill(P.W[s]);
+        uint2 ent = lookup_code<0>(bits[s].hi, l1lane + s * 2 * kTableBytes, P.sub_shift[s]);
+        if (ent.y > 63u) ent = make_uint2(long_code<STAGED>(bits[s], S[s], P.W[s], status), 0u);  // consumed
         x = __fadd_rn(x, __uint_as_float(ent.x));
-        pos[s] += ent.y;
+        bits[s].consume(ent.y);
       }
       out[i] = x;
     }
@@ -490,21 +520,42 @@ __device__ __noinline__ void decode_chunk_global(const StreamState* S, GlobalChu
 template <int KS>
 __global__ void __launch_bounds__(kDecMaxThreads, 1)
 decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, int32_t* __restrict__ status,
-              uint32_t stage_bytes) {
+              const DecodeImage* __restrict__ images, uint32_t stage_bytes) {
   // dynamic shared memory: [pad to 8 KB | 2 tables per stream | StreamState per stream | staging areas]
   extern __shared__ __align__(16) unsigned char s_raw[];
   unsigned char* tables = s_raw + ((kTableBytes - (smem_addr(s_raw) & (kTableBytes - 1))) & (kTableBytes - 1));
   StreamState* S = reinterpret_cast<StreamState*>(s_raw + kTableBytes + KS * 2 * kTableBytes);
-  __shared__ int s_err;
-
+  // the streams were validated and their tables built by decode_prepare_kernel: report a rejected stream (the same
+  // words for every thread) or copy the images in
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
-    const int err = prepare_stream(S[s], tables + s * 2 * kTableBytes, streams.ptr[s], streams.bytes[s], n, &s_err);
+    const int err = images[s].err;
     if (err) {
       if (threadIdx.x == 0) set_status(status, err);
       return;
     }
   }
+#pragma unroll
+  for (int s = 0; s < KS; ++s) {
+    uint2* l1 = reinterpret_cast<uint2*>(tables + s * 2 * kTableBytes);
+    uint2* sub = l1 + kTableBytes / 8;
+    const uint32_t sub_addr = smem_addr(sub);
+    for (uint32_t k = threadIdx.x; k < kTableBytes / 8; k += blockDim.x) {
+      uint2 e = __ldg(&images[s].l1[k]);
+      if (e.y == kLongCode) e.x += sub_addr;
+      l1[k] = e;
+      sub[k] = __ldg(&images[s].sub[k]);
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(&images[s].state);
+    uint4* dst = reinterpret_cast<uint4*>(&S[s]);
+    for (uint32_t k = threadIdx.x; k < sizeof(StreamState) / 16; k += blockDim.x) dst[k] = __ldg(src + k);
+  }
+  __syncthreads();
+  if (threadIdx.x < KS) {
+    S[threadIdx.x].l1 = reinterpret_cast<uint2*>(tables + threadIdx.x * 2 * kTableBytes);
+    S[threadIdx.x].sub = S[threadIdx.x].l1 + kTableBytes / 8;
+  }
+  __syncthreads();
 
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
   unsigned char* stage0 = reinterpret_cast<unsigned char*>(S + KS) + (size_t)warp * KS * stage_bytes;
@@ -572,21 +623,23 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
       if (fits) decode_chunk_fast<KS, true>(S, W, start, base, out, c, lane, next_rows, status);
       else decode_chunk_fast<KS, false>(S, W, start, base, out, c, lane, next_rows, status);
     } else {
-      GlobalChunk G;
+      PartialChunk P;
 #pragma unroll
       for (int s = 0; s < KS; ++s) {
-        G.g[s] = W[s].g;
-        G.nw[s] = W[s].nw;
-        G.start[s] = start[s];
+        P.W[s] = W[s];
+        P.start[s] = start[s];
+        P.sub_shift[s] = 32 - kL1Bits - S[s].sub_bits;
       }
-      decode_chunk_global<KS>(S, G, base, out, c, n, lane, status);
+      const uint32_t l1lane = smem_addr(S[0].l1) | ((lane & (kL1Rep - 1)) * 8u);
+      if (fits) decode_chunk_partial<KS, true>(S, P, l1lane, base, out, c, n, lane, status);
+      else decode_chunk_partial<KS, false>(S, P, l1lane, base, out, c, n, lane, status);
     }
   }
 }
 
 template <int KS>
 cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, uint64_t n, float* out,
-                             int32_t* status, cudaStream_t cs) {
+                             int32_t* status, const DecodeImage* images, cudaStream_t cs) {
   static int sms_of[kMaxDevices] = {};  // by device ordinal; non-zero once the kernel's attributes are set there
   constexpr uint32_t kTables = kTableBytes + KS * (2 * kTableBytes + sizeof(StreamState));
   constexpr uint32_t kMaxDyn = kSmemPerSm - 1024 - kOverrunBytes;  // room for static __shared__ and the padding
@@ -664,19 +717,32 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
     if (cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributePreferredSharedMemoryCarveout, carve) != cudaSuccess)
       return cudaErrorUnknown;
   }
-  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, stage);
+  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, images, stage);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
-                          int32_t* status, cudaStream_t cs) {
+                          int32_t* status, void* images, cudaStream_t cs) {
+  if (k < 1 || k > 4) return cudaErrorInvalidValue;
+  static bool prep_ready[kMaxDevices] = {};  // by device ordinal
+  const int dev = current_device_index();
+  if (dev < 0) return cudaErrorInvalidDevice;
+  if (!prep_ready[dev]) {
+    const cudaError_t e = cudaFuncSetAttribute(decode_prepare_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)kPrepSmem);
+    if (e != cudaSuccess) return e;
+    prep_ready[dev] = true;
+  }
+  DecodeImage* img = static_cast<DecodeImage*>(images);
+  decode_prepare_kernel<<<k, kPrepThreads, kPrepSmem, cs>>>(streams, n, img);
+  if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
   switch (k) {
-    case 1: return launch_decode_ks<1>(base, streams, n, out, status, cs);
-    case 2: return launch_decode_ks<2>(base, streams, n, out, status, cs);
-    case 3: return launch_decode_ks<3>(base, streams, n, out, status, cs);
-    case 4: return launch_decode_ks<4>(base, streams, n, out, status, cs);
+    case 1: return launch_decode_ks<1>(base, streams, n, out, status, img, cs);
+    case 2: return launch_decode_ks<2>(base, streams, n, out, status, img, cs);
+    case 3: return launch_decode_ks<3>(base, streams, n, out, status, img, cs);
+    case 4: return launch_decode_ks<4>(base, streams, n, out, status, img, cs);
     default: return cudaErrorInvalidValue;
   }
 }

@@ -15,9 +15,7 @@ namespace {
 // Largest vector the built-in scratch serves, and the scratch itself. The array lives in every
 // device context that loads the library, from load to exit.
 constexpr uint64_t kNoAllocMaxN = LC_NOALLOC_MAX_N;
-constexpr uint64_t kNoAllocChunks = (kNoAllocMaxN + kChunkElems - 1) / kChunkElems;
-constexpr uint64_t kNoAllocBytes =
-    (sizeof(Control) + 8 * kNoAllocChunks + 255) / 256 * 256 + (kNoAllocChunks * kChunkElems + 255) / 256 * 256;
+constexpr uint64_t kNoAllocBytes = workspace_layout(kNoAllocMaxN).total;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
