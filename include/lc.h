@@ -56,6 +56,7 @@ typedef struct lc_info {
   uint32_t nchunks;
   int32_t valid;           /* 1 if magic, version and constants are those of format version 1 */
   uint32_t fixed_width;    /* 1 if the stream carries fixed-width codes (format section 1.5) */
+  uint32_t shard;          /* 1 if the stream is a shard's, coded with the table of a larger vector (section 1.6) */
 } lc_info;
 
 /* Library version (major*100 + minor). */
@@ -168,6 +169,29 @@ int lc_recover(const float* base, const void* const* streams, const uint64_t* st
 int lc_compress_async(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                       uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs_state,
                       lc_cuda_stream_t cs_side, lc_cuda_event_t state_read);
+
+/*
+ * A vector split over several devices (each holds a contiguous shard of the model state, as under sharded data
+ * parallelism). The method's table, i.e. which buckets priority promotion keeps, their representatives and the
+ * Huffman code (Sections 3.1.1-3.1.2), is a function of the 512 bucket statistics of the WHOLE vector; everything
+ * else is local to a shard. So the pass splits in two around one small exchange:
+ *   1. lc_shard_stats on every shard: the statistics pass; the shard's statistics are left in `stats`.
+ *   2. the caller combines the shards' `stats` buffers, element-wise: bytes [0, 4096) are 512 counts (u64): add;
+ *      bytes [4096, 8192) are 1024 u32 words (running maxima that stand for the buckets' minima and maxima): take
+ *      the maximum, as unsigned numbers. (An all-reduce of 8 KB; every shard must end up with the combined buffer.)
+ *   3. lc_shard_encode on every shard, with the combined statistics: table pass and encode pass. All shards derive
+ *      the same table; each writes a complete stream of its own elements, marked as a shard's (format section 1.6:
+ *      its table lists the shard's own counts, and may give codes to symbols the shard does not use).
+ * lc_recover applies a shard's stream to the shard's part of the base like any other stream; part by part the result
+ * is what the stream of the whole vector would recover, bit for bit.
+ * base, cur, n, nbits, stream, stream_capacity, workspace: as for lc_compress, for the shard; the same workspace in
+ * both calls (the second uses what the first left there). stats / whole_stats: DEVICE, LC_STATS_BYTES, 16-byte aligned.
+ */
+#define LC_STATS_BYTES 8192
+int lc_shard_stats(const float* base, const float* cur, uint64_t n, void* stats, void* workspace,
+                   uint64_t workspace_bytes, lc_cuda_stream_t cs);
+int lc_shard_encode(const float* base, const float* cur, uint64_t n, int nbits, const void* whole_stats, void* stream,
+                    uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs);
 
 /*
  * Checkpoint merging (Section 3.2, "Checkpoint Merging"): the k streams that lead from `base` to a later tracked

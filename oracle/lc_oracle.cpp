@@ -194,7 +194,8 @@ struct Table {
   int nbits = 0;
   int nsym = 1;
   int max_len = 0;
-  int fixed = 0;  // 1: fixed-width codes (format section 1.5) instead of the Huffman code
+  int fixed = 0;   // 1: fixed-width codes (format section 1.5) instead of the Huffman code
+  int shared = 0;  // 1: the table was built from a larger vector than the stream codes (format section 1.6)
   int key[512] = {};
   int len[512] = {};
   float rep[512] = {};
@@ -333,8 +334,8 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   if (!(s[0] == 'L' && s[1] == 'C' && s[2] == 'C' && s[3] == '1')) return LCO_ERR_FORMAT;
   if (get_le(s + 4, 2) != 1) return LCO_ERR_FORMAT;
   const int nbits = static_cast<int>(s[6]);
-  if (nbits < 1 || nbits > 9 || s[7] > 1) return LCO_ERR_FORMAT;
-  const int fixed = static_cast<int>(s[7]);
+  if (nbits < 1 || nbits > 9 || s[7] > 3) return LCO_ERR_FORMAT;
+  const int fixed = static_cast<int>(s[7] & 1), shared = static_cast<int>(s[7] >> 1);
   const uint64_t n = get_le(s + 8, 8);
   const uint64_t nsym = get_le(s + 16, 4);
   const uint64_t max_len = get_le(s + 20, 4);
@@ -365,7 +366,7 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
     p.table.rep[j] = bits_float(static_cast<uint32_t>(get_le(e + 4, 4)));
     p.table.count[j] = get_le(e + 8, 8);
     if (e[3] != 0 || p.table.len[j] > 63) return LCO_ERR_FORMAT;
-    if (!fixed && p.table.count[j] == 0 && p.table.len[j] != 0) return LCO_ERR_FORMAT;
+    if (!fixed && !shared && p.table.count[j] == 0 && p.table.len[j] != 0) return LCO_ERR_FORMAT;
     if (p.table.count[j] > 0) used += 1;
     count_sum += p.table.count[j];
     bit_sum += p.table.count[j] * static_cast<uint64_t>(p.table.len[j]);
@@ -375,6 +376,7 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
     return LCO_ERR_FORMAT;
   p.table.max_len = seen_max;
   p.table.fixed = fixed;
+  p.table.shared = shared;
   if (fixed) {
     int width = 0;
     while ((1ull << width) < nsym) width += 1;
@@ -382,11 +384,15 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
       if (p.table.len[j] != width) return LCO_ERR_FORMAT;
       p.table.code[j] = j;
     }
-  } else if (used >= 2) {
-    // Kraft equality, as an exact integer sum of 2^(63-len).
+  } else if (shared ? seen_max != 0 : used >= 2) {
+    // Kraft equality, as an exact integer sum of 2^(63-len), over the symbols that have a code: the used ones,
+    // and with a shared table also those that only other parts of the larger vector use.
     unsigned __int128 kraft = 0;
     for (uint64_t j = 0; j < nsym; ++j) {
-      if (p.table.count[j] == 0) continue;
+      if (shared ? p.table.len[j] == 0 : p.table.count[j] == 0) {
+        if (p.table.count[j] != 0) return LCO_ERR_FORMAT;
+        continue;
+      }
       if (p.table.len[j] == 0) return LCO_ERR_FORMAT;
       kraft += static_cast<unsigned __int128>(1) << (63 - p.table.len[j]);
     }
@@ -507,7 +513,7 @@ void write_header_and_table(uint8_t* stream, const Table& t, uint64_t n, int nbi
   h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
   put_le(h + 4, 1, 2);
   h[6] = static_cast<uint8_t>(nbits);
-  h[7] = static_cast<uint8_t>(t.fixed);
+  h[7] = static_cast<uint8_t>(t.fixed | (t.shared << 1));
   put_le(h + 8, n, 8);
   put_le(h + 16, static_cast<uint64_t>(t.nsym), 4);
   put_le(h + 20, static_cast<uint64_t>(t.max_len), 4);
@@ -845,6 +851,46 @@ int lco_recover_mt(const float* base, const uint8_t* const* streams, const uint6
     for (int th = 0; th < nthreads; ++th)
       if (status[th] != LCO_OK) return status[th];
   }
+  return LCO_OK;
+}
+
+
+// One shard of a vector that is split over several devices (format section 1.6): the table (kept buckets,
+// representatives, code) comes from the statistics of the WHOLE vector [0, n_total), which every shard obtains by
+// exchanging its 512 bucket statistics (counts add, minima and maxima combine), so all shards code with the same
+// table; the stream codes the elements [lo, hi) only, as a vector of hi - lo elements, and its table lists the
+// shard's own counts. Recovering every shard's stream over its part of the base gives, part by part, what the
+// stream of the whole vector recovers.
+int lco_compress_shard(const float* base, const float* cur, uint64_t n_total, uint64_t lo, uint64_t hi, int nbits,
+                       uint8_t* stream, uint64_t capacity, uint64_t* out_bytes) {
+  if (nbits < 1 || nbits > 9 || n_total >= (1ull << 32) || lo > hi || hi > n_total) return LCO_ERR_ARG;
+  const uint64_t n = hi - lo;
+  if (capacity < stream_bound(n, nbits)) return LCO_ERR_CAPACITY;
+  std::vector<Bucket> buckets(512);
+  delta_buckets(base, cur, n_total, buckets.data());
+  Table t;
+  Selection sel;
+  const int rc = build_table(buckets.data(), n_total, nbits, &t, &sel);
+  if (rc != LCO_OK) return rc;
+  t.shared = 1;
+  for (int j = 0; j < t.nsym; ++j) t.count[j] = 0;
+  for (uint64_t i = lo; i < hi; ++i) t.count[sel.symbol_of_key[bucket_key(cur[i] - base[i])]] += 1;
+
+  const Layout L = layout_for(n, t.nsym);
+  std::memset(stream, 0, L.payload_off);
+  uint8_t* chunk_index = stream + L.chunk_index_off;
+  uint8_t* lane_index = stream + L.lane_index_off;
+  uint64_t payload_bytes = 0, payload_bits = 0;
+  for (uint64_t c = 0; c < L.nchunks; ++c) {
+    put_le(chunk_index + 8 * c, payload_bytes, 8);
+    uint64_t chunk_bits = 0;
+    payload_bytes += encode_chunk(base + lo, cur + lo, n, t, sel, c, lane_index + 2 * kLanes * c,
+                                  stream + L.payload_off + payload_bytes, &chunk_bits);
+    payload_bits += chunk_bits;
+  }
+  put_le(chunk_index + 8 * L.nchunks, payload_bytes, 8);
+  write_header_and_table(stream, t, n, nbits, L, payload_bits, payload_bytes);
+  *out_bytes = L.payload_off + payload_bytes;
   return LCO_OK;
 }
 

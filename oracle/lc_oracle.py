@@ -38,6 +38,7 @@ def lib():
         L.lco_table_mode.argtypes = [vp, vp, u64, i32, i32, vp, vp, vp, vp, vp]
         L.lco_compress_mode.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_mode_mt.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64), i32]
+        L.lco_compress_shard.argtypes = [vp, vp, u64, u64, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_mt.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), i32]
         L.lco_recover_mt.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, i32]
@@ -131,6 +132,19 @@ def compress(base, cur, nbits, threads=None, fixed=False):
     else:
         rc = lib().lco_compress_mode_mt(pb, pc, base.size, nbits, int(bool(fixed)), buf.ctypes.data, cap,
                                         C.byref(out), int(threads))
+    if rc < 0:
+        raise OracleError(rc)
+    return buf[: out.value].copy()
+
+
+def compress_shard(base, cur, lo, hi, nbits):
+    """Stream of the elements [lo, hi) coded with the table of the whole vector (a shard of a split vector)."""
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    cap = stream_bound(hi - lo, nbits)
+    buf = np.zeros(cap, np.uint8)
+    out = C.c_uint64(0)
+    rc = lib().lco_compress_shard(pb, pc, base.size, lo, hi, nbits, buf.ctypes.data, cap, C.byref(out))
     if rc < 0:
         raise OracleError(rc)
     return buf[: out.value].copy()

@@ -18,7 +18,7 @@ MAX_CHAIN = 8
 
 SYMBOLS = (
     "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_update", "lc_compress_timed",
-    "lc_recover", "lc_compress_opt", "lc_debug_compress_wait", "lc_merge", "lc_compress_async",
+    "lc_recover", "lc_compress_opt", "lc_debug_compress_wait", "lc_merge", "lc_compress_async", "lc_shard_stats", "lc_shard_encode",
     "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
     "lc_debug_bins", "lc_debug_codes", "lc_compress_noalloc",
 )
@@ -29,7 +29,7 @@ class LCInfo(C.Structure):
     _fields_ = [
         ("n", C.c_uint64), ("total_bytes", C.c_uint64), ("payload_bits", C.c_uint64),
         ("payload_offset", C.c_uint64), ("nbits", C.c_uint32), ("nsym", C.c_uint32),
-        ("max_len", C.c_uint32), ("nchunks", C.c_uint32), ("valid", C.c_int32), ("fixed_width", C.c_uint32),
+        ("max_len", C.c_uint32), ("nchunks", C.c_uint32), ("valid", C.c_int32), ("fixed_width", C.c_uint32), ("shard", C.c_uint32),
     ]
 
 
@@ -69,6 +69,8 @@ def lib():
     L.lc_compress_timed.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, C.POINTER(C.c_float)]
     L.lc_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
     L.lc_compress_async.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, vp, vp]
+    L.lc_shard_stats.argtypes = [vp, vp, u64, vp, vp, u64, vp]
+    L.lc_shard_encode.argtypes = [vp, vp, u64, i32, vp, vp, u64, vp, u64, vp]
     L.lc_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, vp, vp, u64, vp]
     L.lc_stream_info.argtypes = [vp, C.POINTER(LCInfo), vp]
     L.lc_last_status.argtypes = [vp, vp]
@@ -241,6 +243,57 @@ def compress_two_streams(base, cur, nbits, stream, workspace, state_stream, side
                                  C.c_void_p(state_stream.cuda_stream), C.c_void_p(side_stream.cuda_stream),
                                  C.c_void_p(state_read.cuda_event))
     _check(rc, "lc_compress_async")
+
+
+STATS_BYTES = 8192
+
+
+def shard_stats(base, cur, workspace, stats=None):
+    """lc_shard_stats: the statistics pass of one shard; returns the 8 KB statistics buffer (uint8 tensor)."""
+    _f32_cuda(base, "base"), _f32_cuda(cur, "cur")
+    if stats is None:
+        stats = torch.empty(STATS_BYTES, dtype=torch.uint8, device=base.device)
+    _check(lib().lc_shard_stats(base.data_ptr(), cur.data_ptr(), base.numel(), stats.data_ptr(), workspace.data_ptr(),
+                                workspace.numel(), _cs(base.device)), "lc_shard_stats")
+    return stats
+
+
+def combine_stats(buffers):
+    """Element-wise combination of shards' statistics buffers on one device (what an all-reduce over the shards
+    computes): counts add, the two running-maximum arrays take the unsigned maximum."""
+    counts = torch.stack([b[:4096].view(torch.int64) for b in buffers]).sum(0)
+    # unsigned 32-bit maximum through int64 (the words can have their top bit set)
+    words = torch.stack([b[4096:].view(torch.int32).to(torch.int64) & 0xFFFFFFFF for b in buffers]).amax(0)
+    out = torch.empty_like(buffers[0])
+    out[:4096] = counts.view(torch.uint8)
+    out[4096:] = words.to(torch.int32).view(torch.uint8)  # truncation keeps the low 32 bits
+    return out
+
+
+def all_reduce_stats(stats, group=None):
+    """The exchange between lc_shard_stats and lc_shard_encode over a torch.distributed group: after it every rank
+    holds the statistics of the whole vector. Two small all-reduces (512 sums, 1024 maxima)."""
+    import torch.distributed as dist
+
+    counts = stats[:4096].view(torch.int64).clone()
+    words = stats[4096:].view(torch.int32).to(torch.int64) & 0xFFFFFFFF  # unsigned values in a signed type
+    dist.all_reduce(counts, op=dist.ReduceOp.SUM, group=group)
+    dist.all_reduce(words, op=dist.ReduceOp.MAX, group=group)
+    stats[:4096] = counts.view(torch.uint8)
+    stats[4096:] = words.to(torch.int32).view(torch.uint8)  # truncation keeps the low 32 bits
+    return stats
+
+
+def shard_encode(base, cur, nbits, whole_stats, workspace, stream=None):
+    """lc_shard_encode: table and encode pass of one shard with the whole vector's statistics; returns the stream."""
+    n = base.numel()
+    if stream is None:
+        stream = alloc_stream(n, nbits, base.device)
+    _check(lib().lc_shard_encode(base.data_ptr(), cur.data_ptr(), n, nbits, whole_stats.data_ptr(), stream.data_ptr(),
+                                 stream.numel(), workspace.data_ptr(), workspace.numel(), _cs(base.device)),
+           "lc_shard_encode")
+    _check(last_status(workspace), "lc_shard_encode (device)")
+    return stream[: stream_info(stream).total_bytes]
 
 
 def merge_async(base, streams, nbits, stream, scratch, workspace):

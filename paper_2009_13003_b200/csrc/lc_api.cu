@@ -1,4 +1,5 @@
 // C ABI entry points (declared in include/lc.h): argument checks, workspace carving, launch order.
+#include <stddef.h>
 #include <string.h>
 
 #include "lc_common.cuh"
@@ -43,7 +44,7 @@ int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, vo
   cudaError_t e = cudaMemsetAsync(static_cast<uint8_t*>(workspace) + skip, 0, W.plane_off - skip, cs);
   if (e != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, opt.fixed_width, cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, opt.fixed_width, nullptr, cs)) != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), tracked_out, opt,
                          cs)) != cudaSuccess)
     return LC_ERR_CUDA;
@@ -142,7 +143,7 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
   ok = ok && cudaEventRecord(ev[0], cs) == cudaSuccess;
   ok = ok && launch_stats(base, cur, n, c.ctl, c.plane, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[1], cs) == cudaSuccess;
-  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, false, cs) == cudaSuccess;
+  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, false, nullptr, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[2], cs) == cudaSuccess;
   ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[3], cs) == cudaSuccess;
@@ -196,10 +197,47 @@ int lc_compress_async(const float* base, const float* cur, uint64_t n, int nbits
   if (cudaEventRecord(state_read, cs_state) != cudaSuccess) return LC_ERR_CUDA;
   // beside whatever cs_state does next: table and encode, which work on the bucket statistics and the key plane
   if (cudaStreamWaitEvent(cs_side, state_read, 0) != cudaSuccess) return LC_ERR_CUDA;
-  if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), /*wide_ok=*/false, false, cs_side) != cudaSuccess)
+  if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), /*wide_ok=*/false, false, nullptr, cs_side) != cudaSuccess)
     return LC_ERR_CUDA;
   if (launch_encode(c.ctl, c.tiles, c.plane, nullptr, nullptr, n, static_cast<uint8_t*>(stream), nullptr,
                     EncodeOptions(), cs_side) != cudaSuccess)
+    return LC_ERR_CUDA;
+  return LC_OK;
+}
+
+int lc_shard_stats(const float* base, const float* cur, uint64_t n, void* stats, void* workspace,
+                   uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+  if (n >= (1ull << 32) || !stats || !workspace || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
+  if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stats, 16) || !aligned(workspace, 256)) return LC_ERR_ARG;
+  const WorkspaceLayout W = workspace_layout(n);
+  if (workspace_bytes < W.total) return LC_ERR_CAPACITY;
+  const Carved c = carve(workspace, W);
+  if (cudaMemsetAsync(workspace, 0, W.plane_off, cs) != cudaSuccess) return LC_ERR_CUDA;
+  if (launch_stats(base, cur, n, c.ctl, c.plane, cs) != cudaSuccess) return LC_ERR_CUDA;
+  // count, inv_min, max_bits: contiguous in the control block, in ShardStats' order
+  static_assert(offsetof(Control, inv_min) - offsetof(Control, count) == offsetof(ShardStats, inv_min) &&
+                    offsetof(Control, max_bits) - offsetof(Control, count) == offsetof(ShardStats, max_bits),
+                "one copy moves the three arrays");
+  if (cudaMemcpyAsync(stats, c.ctl->count, sizeof(ShardStats), cudaMemcpyDeviceToDevice, cs) != cudaSuccess)
+    return LC_ERR_CUDA;
+  return LC_OK;
+}
+
+int lc_shard_encode(const float* base, const float* cur, uint64_t n, int nbits, const void* whole_stats, void* stream,
+                    uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+  if (nbits < 1 || nbits > kMaxNbits || n >= (1ull << 32)) return LC_ERR_ARG;
+  if (!stream || !workspace || !whole_stats || (n > 0 && (!base || !cur))) return LC_ERR_ARG;
+  if (!aligned(base, 16) || !aligned(cur, 16) || !aligned(stream, 16) || !aligned(whole_stats, 16) ||
+      !aligned(workspace, 256))
+    return LC_ERR_ARG;
+  const WorkspaceLayout W = workspace_layout(n);
+  if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
+  const Carved c = carve(workspace, W);
+  if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, false,
+                   static_cast<const ShardStats*>(whole_stats), cs) != cudaSuccess)
+    return LC_ERR_CUDA;
+  if (launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(),
+                    cs) != cudaSuccess)
     return LC_ERR_CUDA;
   return LC_OK;
 }
@@ -234,6 +272,7 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
   memset(info, 0, sizeof *info);
   info->nbits = h[6];
   info->fixed_width = h[7] & 1u;
+  info->shard = (h[7] >> 1) & 1u;
   info->n = le(8, 8);
   info->nsym = (uint32_t)le(16, 4);
   info->max_len = (uint32_t)le(20, 4);
@@ -241,7 +280,7 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
   info->payload_bits = le(40, 8);
   info->total_bytes = le(48, 8);
   info->payload_offset = le(56, 8);
-  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 && h[7] <= 1 &&
+  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 && h[7] <= 3 &&
                  le(24, 4) == kChunkElems && le(28, 2) == kLanes && le(30, 2) == kGroup &&
                  le(36, 4) == kPayloadAlign)
                     ? 1

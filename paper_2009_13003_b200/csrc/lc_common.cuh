@@ -80,6 +80,14 @@ struct Control {
   uint32_t max_bits[kKeys];         // max over the bucket of bits
   EncEntry enc[kKeys];
 };
+// The bucket statistics as a shard of a split vector hands them out and takes them back (include/lc.h, lc_shard_*):
+// the three arrays of Control, in Control's order, so that one copy moves them.
+struct ShardStats {
+  unsigned long long count[kKeys];
+  uint32_t inv_min[kKeys];
+  uint32_t max_bits[kKeys];
+};
+static_assert(sizeof(ShardStats) == LC_STATS_BYTES, "size promised by the header");
 static_assert(sizeof(Control) % 256 == 0, "control block must keep the planes 256-byte aligned");
 
 // lc_recover keeps the decode tables of the (at most four) streams of one launch behind the control block, at an
@@ -133,8 +141,10 @@ cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Contro
 // wide_ok: false if the encode pass will not be able to read base and cur (the table pass then rejects a vector
 // with an exponent field >= 128 with LC_ERR_RANGE)
 // fixed: fixed-width codes (format section 1.5) instead of the Huffman code
+// whole: nullptr, or the statistics of the whole vector of which this call codes a shard (format section 1.6):
+//        kept buckets, representatives and code then come from them, the table's counts from ctl's own
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, bool fixed,
-                         cudaStream_t cs);
+                         const ShardStats* whole, cudaStream_t cs);
 // tracked_out: nullptr, or where to write base + quantized delta (may be base itself)
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
                           const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, const EncodeOptions& opt,

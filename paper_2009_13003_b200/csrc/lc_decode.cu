@@ -70,6 +70,7 @@ struct alignas(16) StreamState {
   unsigned long long chunk_index_off, lane_index_off;
   uint32_t nsym, max_len, nchunks, only_rep;
   uint32_t fixed;  // fixed-width codes (format section 1.5): every symbol is coded, used or not
+  uint32_t shared_table;  // the table comes from a larger vector (format section 1.6): unused symbols may have codes
   // validation accumulators
   unsigned long long kraft, count_sum, bit_sum;
   uint32_t seen_max, nused, nsub;
@@ -120,7 +121,8 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
       S.payload_off = load_le(h + 56, 8);
       const bool magic = h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1';
       S.fixed = h[7] & 1u;
-      if (!magic || load_le(h + 4, 2) != 1 || nbits < 1 || nbits > (uint32_t)kMaxNbits || h[7] > 1) err = LC_ERR_FORMAT;
+      S.shared_table = (h[7] >> 1) & 1u;
+      if (!magic || load_le(h + 4, 2) != 1 || nbits < 1 || nbits > (uint32_t)kMaxNbits || h[7] > 3) err = LC_ERR_FORMAT;
       else if (S.nsym < 1 || S.nsym > (1u << nbits) || S.max_len > 63) err = LC_ERR_FORMAT;
       else if (load_le(h + 24, 4) != kChunkElems || load_le(h + 28, 2) != kLanes ||
                load_le(h + 30, 2) != kGroup || load_le(h + 36, 4) != kPayloadAlign) err = LC_ERR_FORMAT;
@@ -148,7 +150,7 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
 
   // ---- table entries: a thread per symbol (up to 509 symbols, CTAs of 256 threads and more)
   const uint32_t nsym = S.nsym;
-  const bool fixed = S.fixed != 0;
+  const bool fixed = S.fixed != 0, shared_table = S.shared_table != 0;
   uint32_t fixed_width = 0;
   while ((1u << fixed_width) < nsym) fixed_width += 1;
   bool entry_bad = false;
@@ -157,16 +159,19 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
     const uint32_t my_len = (e.x >> 16) & 255u, my_rep = e.y;
     const unsigned long long my_count = ((unsigned long long)e.w << 32) | e.z;
     entry_bad |= (e.x >> 24) != 0 || my_len > 63;
-    entry_bad |= fixed ? (my_len != fixed_width) : (my_count == 0 && my_len != 0);
+    entry_bad |= fixed ? (my_len != fixed_width) : (!shared_table && my_count == 0 && my_len != 0);
+    entry_bad |= my_count != 0 && my_len == 0 && shared_table && S.max_len != 0;  // a used symbol needs its code
     S.sym_len[sym] = (uint8_t)my_len;
+    atomicMax(&S.seen_max, my_len);
     if (my_count != 0) {
       atomicAdd(&S.count_sum, my_count);
       atomicAdd(&S.bit_sum, my_count * my_len);
-      atomicMax(&S.seen_max, my_len);
     }
-    if (fixed ? (fixed_width > 0 || sym == 0) : (my_count != 0)) {  // the symbols that have a code
+    if (!fixed && my_count != 0) S.only_rep = my_rep;  // meaningful only when no symbol has a code length
+    if (fixed ? (fixed_width > 0 || sym == 0) : (shared_table && S.max_len != 0 ? my_len != 0 : my_count != 0)) {
+      // the symbols that have a code
       atomicAdd(&S.nused, 1u);
-      if (fixed ? sym == 0 : true) S.only_rep = my_rep;  // meaningful only when a single symbol is coded
+      if (fixed && sym == 0) S.only_rep = my_rep;
       if (my_len > 0 && my_len <= 63) {
         atomicAdd(&S.kraft, 1ull << (63 - my_len));
         atomicAdd(&S.len_count[my_len], 1u);

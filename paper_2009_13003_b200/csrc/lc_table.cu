@@ -21,7 +21,7 @@ __device__ __forceinline__ void store_le(uint8_t* p, uint64_t v, int bytes) {
 
 __global__ void __launch_bounds__(kTableThreads)
 table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restrict__ stream, int wide_ok,
-             int fixed) {
+             int fixed, const ShardStats* __restrict__ whole) {
   __shared__ uint32_t warp_cand[16];
   __shared__ uint16_t sym_of_key[kKeys];
   __shared__ unsigned long long sym_count[kMaxSym];
@@ -39,6 +39,12 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
 
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
+  // The statistics that decide the table: this vector's own, or those of the whole vector it is a shard of.
+  const unsigned long long* g_count = whole ? whole->count : ctl->count;
+  const uint32_t* g_inv_min = whole ? whole->inv_min : ctl->inv_min;
+  const uint32_t* g_max_bits = whole ? whole->max_bits : ctl->max_bits;
+  __shared__ unsigned long long s_whole_total;
+  __shared__ unsigned long long sym_local[kMaxSym];  // the table's counts: this vector's own elements per symbol
 
   // ---- an earlier pass of the same call has failed (lc_merge: a stream was rejected): leave no stream behind
   if (ctl->status != 0) {  // nothing in this kernel has written the word yet: the same for every thread
@@ -47,7 +53,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   }
 
   // ---- non-finite deltas make the vector unencodable ------------------------------------------
-  const bool bad = (tid == 255 || tid == 511) && ctl->count[tid] != 0;
+  const bool bad = (tid == 255 || tid == 511) && g_count[tid] != 0;
   if (__syncthreads_or(bad)) {
     if (tid == 0) {
       set_status(&ctl->status, LC_ERR_NONFINITE);
@@ -57,7 +63,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   }
 
   // ---- does the one-byte key plane identify every bucket? (only if all exponent fields are < 128)
-  const bool big = (tid & 255) >= 128 && ctl->count[tid] != 0;
+  const bool big = (tid & 255) >= 128 && (g_count[tid] != 0 || ctl->count[tid] != 0);
   const int wide = __syncthreads_or(big);
   if (wide && !wide_ok) {
     // the caller has released base and cur, and the one-byte keys do not identify the buckets of this vector
@@ -76,7 +82,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   if (tid < 508) {
     const uint32_t E = 254 - (tid >> 1), s = tid & 1;
     key = 256 * s + E;
-    cnt = ctl->count[key];
+    cnt = g_count[key];
     cand = cnt != 0;
   }
   if (tid < kMaxSym) {
@@ -91,7 +97,9 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     s_kept_total = 0;
     s_payload_bits = 0;
     s_maxlen = 0;
+    s_whole_total = 0;
   }
+  sym_local[tid] = 0;
   const uint32_t ballot = __ballot_sync(0xffffffffu, cand);
   if (lane == 0) warp_cand[warp] = __popc(ballot);
   __syncthreads();
@@ -109,17 +117,22 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     sym_count[sym] = cnt;
     sym_key[sym] = key;
     // midrange of two values with the same sign and exponent, rounded to nearest even, on mantissas.
-    const uint32_t mmin = (~ctl->inv_min[key]) & 0x7FFFFFu;
-    const uint32_t mmax = ctl->max_bits[key] & 0x7FFFFFu;
+    sym_local[sym] = ctl->count[key];
+    const uint32_t mmin = (~g_inv_min[key]) & 0x7FFFFFu;
+    const uint32_t mmax = g_max_bits[key] & 0x7FFFFFu;
     const uint32_t t = mmin + mmax;
     uint32_t mr = t >> 1;
     if ((t & 1u) && (mr & 1u)) mr += 1;
     sym_rep[sym] = (key << 23) | mr;
     atomicAdd(&s_kept_total, cnt);
   }
+  if (whole) atomicAdd(&s_whole_total, g_count[tid]);  // elements of the whole vector
   __syncthreads();
   if (tid == 0) {
-    sym_count[0] = n - s_kept_total;
+    sym_count[0] = (whole ? s_whole_total : n) - s_kept_total;
+    unsigned long long kept_local = 0;
+    for (uint32_t j = 1; j < nsym; ++j) kept_local += sym_local[j];
+    sym_local[0] = n - kept_local;
   }
   __syncthreads();
 
@@ -212,6 +225,12 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   }
   __syncthreads();
 
+  // ---- payload size: this vector's own elements, with the lengths just found --------------------------
+  if (tid == 0) s_payload_bits = 0;
+  __syncthreads();
+  if (tid < (int)nsym) atomicAdd(&s_payload_bits, sym_local[tid] * sym_len[tid]);
+  __syncthreads();
+
   // ---- outputs ---------------------------------------------------------------------------------------
   {
     const uint32_t sym = sym_of_key[tid];
@@ -229,7 +248,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     e[2] = (uint8_t)sym_len[tid];
     e[3] = 0;
     store_le(e + 4, sym_rep[tid], 4);
-    store_le(e + 8, sym_count[tid], 8);
+    store_le(e + 8, sym_local[tid], 8);
   }
   if (tid == 0) {
     ctl->nsym = nsym;
@@ -240,7 +259,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
     store_le(h + 4, 1, 2);
     h[6] = (uint8_t)nbits;
-    h[7] = (uint8_t)(fixed ? 1 : 0);
+    h[7] = (uint8_t)((fixed ? 1 : 0) | (whole ? 2 : 0));
     store_le(h + 8, n, 8);
     store_le(h + 16, nsym, 4);
     store_le(h + 20, s_maxlen, 4);
@@ -264,8 +283,8 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
 }  // namespace
 
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, bool fixed,
-                         cudaStream_t cs) {
-  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0, fixed ? 1 : 0);
+                         const ShardStats* whole, cudaStream_t cs) {
+  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0, fixed ? 1 : 0, whole);
   return cudaGetLastError();
 }
 

@@ -58,6 +58,9 @@ MUTATIONS = [
      "const uint64_t lo = c * kChunkElems, hi = std::min(n, lo + kChunkElems - 1);\n        if (parsed[j].table.max_len == 0)"),
     ("fixed width one bit short", "while ((1 << width) < t->nsym) width += 1;", "while ((2 << width) < t->nsym) width += 1;"),
     ("fixed-width code is not the symbol id", "t->code[j] = static_cast<uint64_t>(j);", "t->code[j] = static_cast<uint64_t>(t->nsym - 1 - j);"),
+    ("shard codes from the vector's first element", "payload_bytes += encode_chunk(base + lo, cur + lo, n, t, sel, c,", "payload_bytes += encode_chunk(base, cur, n, t, sel, c,"),
+    ("shard's table built from the shard alone", "delta_buckets(base, cur, n_total, buckets.data());\n  Table t;\n  Selection sel;\n  const int rc = build_table(buckets.data(), n_total, nbits, &t, &sel);\n  if (rc != LCO_OK) return rc;\n  t.shared = 1;",
+     "delta_buckets(base + lo, cur + lo, hi - lo, buckets.data());\n  Table t;\n  Selection sel;\n  const int rc = build_table(buckets.data(), hi - lo, nbits, &t, &sel);\n  if (rc != LCO_OK) return rc;\n  t.shared = 1;"),
     ("size model uses floor log", "while ((1ull << width) < k) width += 1;", "while ((2ull << width) <= k) width += 1;"),
 ]
 
@@ -87,6 +90,7 @@ class _Oracle:
         L.lco_midrange.argtypes = [C.c_float, C.c_float]
         L.lco_midrange.restype = C.c_float
         L.lco_compress_mode.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64)]
+        L.lco_compress_shard.argtypes = [vp, vp, u64, u64, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_apply_quantized.argtypes = [vp, vp, u64, i32, vp]
         L.lco_compress_chunks.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
         L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
@@ -100,6 +104,14 @@ class _Oracle:
         out = C.c_uint64(0)
         assert self.L.lco_compress_mode(base.ctypes.data, cur.ctypes.data, base.size, nbits, 1, buf.ctypes.data, cap,
                                         C.byref(out)) == 0
+        return buf[: out.value].copy()
+
+    def compress_shard(self, base, cur, lo, hi, nbits):
+        cap = int(self.L.lco_stream_bound(hi - lo, nbits))
+        buf = np.zeros(cap + 64, np.uint8)
+        out = C.c_uint64(0)
+        assert self.L.lco_compress_shard(base.ctypes.data, cur.ctypes.data, base.size, lo, hi, nbits, buf.ctypes.data, cap,
+                                         C.byref(out)) == 0
         return buf[: out.value].copy()
 
     def apply_quantized(self, base, cur, nbits):
@@ -275,6 +287,16 @@ def _pins_hold(o):
         ids = [order.index(k) + 1 for k in keys]
         want_bits = "".join(format(i, "03b") for i in ids).ljust(32, "0")
         if word0 != int(want_bits, 2):
+            return False
+        # a shard of the vector, coded with the whole vector's table, recovers its part of what the whole stream recovers
+        ss = o.compress_shard(base, cur, 4096, n, 3)
+        if not np.array_equal(o.recover(base[4096:], [ss]).view(np.uint32), once[4096:].view(np.uint32)):
+            return False
+        d2 = cur.copy()
+        d2[:3000] = base[:3000] + (cur[:3000] - base[:3000]) * 1024  # the first part now holds all the large deltas
+        whole2 = o.recover(base, [o.compress(base, d2, 2)])
+        s2b = o.compress_shard(base, d2, 3000, n, 2)
+        if not np.array_equal(o.recover(base[3000:], [s2b]).view(np.uint32), whole2[3000:].view(np.uint32)):
             return False
         # the threaded timing mode writes the same bytes and states
         if o.compress_mt(base, cur, 3, 3).tobytes() != s.tobytes():

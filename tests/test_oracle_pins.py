@@ -415,7 +415,7 @@ def test_reader_rejects_corruption(oracle):
     expect(setb(0, ord("X")), oracle.ERR_FORMAT)     # magic
     expect(setb(4, 2), oracle.ERR_FORMAT)            # version
     expect(setb(6, 10), oracle.ERR_FORMAT)           # nbits
-    expect(setb(7, 2), oracle.ERR_FORMAT)            # flags
+    expect(setb(7, 4), oracle.ERR_FORMAT)            # flags
     expect(setb(16, 200), oracle.ERR_FORMAT)         # nsym > 2^nbits
     expect(setb(24, 1), oracle.ERR_FORMAT)           # chunk_elems
     expect(setb(64 + 16 + 2, 1), oracle.ERR_FORMAT)  # a code length changed: Kraft / payload_bits
@@ -657,3 +657,55 @@ def test_reader_checks_fixed_width_streams(oracle):
         with pytest.raises(oracle.OracleError) as e:
             oracle.recover(base, [s])
         assert e.value.code == oracle.ERR_FORMAT
+
+
+# ---------------------------------------------------------------- shards of a split vector (format section 1.6)
+
+
+def test_shards_code_with_the_whole_vectors_table(oracle):
+    rng = np.random.default_rng(101)
+    n = 5 * 4096 + 321
+    base, cur = _random_case(rng, n)
+    cur[3 * 4096:] = base[3 * 4096:] + (cur[3 * 4096:] - base[3 * 4096:]) * 64  # the parts differ in scale
+    nbits = 3
+    whole = oracle.compress(base, cur, nbits)
+    pw = _parse(whole)
+    sym = oracle.symbols(base, cur, nbits)
+    want = oracle.recover(base, [whole])
+    cuts = [0, 2 * 4096, 3 * 4096, n]  # chunk-aligned cuts
+    counts = np.zeros(pw["nsym"], np.uint64)
+    for lo, hi in zip(cuts[:-1], cuts[1:]):
+        s = oracle.compress_shard(base, cur, lo, hi, nbits)
+        p = _parse(s)
+        assert p["flags"] == 2 and p["n"] == hi - lo
+        # the same table as the whole vector's, but for the counts, which are the shard's own
+        for f in ("key", "len", "rep"):
+            assert np.array_equal(p["tab"][f], pw["tab"][f])
+        assert np.array_equal(p["tab"]["count"], np.bincount(sym[lo:hi], minlength=pw["nsym"]).astype(np.uint64))
+        counts += p["tab"]["count"]
+        # its symbols, its chunks and its recovered part are the whole stream's
+        assert np.array_equal(oracle.decode_symbols(s, hi - lo), sym[lo:hi])
+        c0 = lo // 4096
+        for c in range(p["nchunks"]):
+            assert np.array_equal(p["lane_bits"][c], pw["lane_bits"][c0 + c])
+            a = s[p["po"] + int(p["chunk_off"][c]): p["po"] + int(p["chunk_off"][c + 1])]
+            b = whole[pw["po"] + int(pw["chunk_off"][c0 + c]): pw["po"] + int(pw["chunk_off"][c0 + c + 1])]
+            assert a.tobytes() == b.tobytes()
+        out = oracle.recover(base[lo:hi], [s])
+        assert np.array_equal(out.view(np.uint32), want[lo:hi].view(np.uint32))
+    assert np.array_equal(counts, pw["tab"]["count"])
+    # a single shard that is the whole vector: the whole vector's stream but for the flag
+    one = oracle.compress_shard(base, cur, 0, n, nbits)
+    one[7] = 0
+    assert one.tobytes() == whole.tobytes()
+    # a cut inside a chunk: other chunks, the same symbols and state
+    s = oracle.compress_shard(base, cur, 1000, 9000, nbits)
+    assert np.array_equal(oracle.decode_symbols(s, 8000), sym[1000:9000])
+    assert np.array_equal(oracle.recover(base[1000:9000], [s]).view(np.uint32), want[1000:9000].view(np.uint32))
+    # the flag is what allows codes for symbols the shard does not use
+    unused = oracle.compress_shard(base, cur, 0, 4096, 8)
+    if np.any((_parse(unused)["tab"]["count"] == 0) & (_parse(unused)["tab"]["len"] != 0)):
+        bad = unused.copy()
+        bad[7] = 0
+        with pytest.raises(oracle.OracleError):
+            oracle.recover(base[:4096], [bad])
