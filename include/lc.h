@@ -236,7 +236,11 @@ int lc_compress_host(const float* base_host, const float* cur_host, uint64_t n, 
                      void* stream_host, uint64_t stream_capacity, uint64_t* stream_bytes_out,
                      void* arena, uint64_t arena_bytes, lc_cuda_stream_t cs);
 
-/* base_host HOST fp32[n]; streams_host HOST array of k HOST pointers; out_host HOST fp32[n]. */
+/* base_host HOST fp32[n]; streams_host HOST array of k HOST pointers; out_host HOST fp32[n]. A vector of 128
+ * chunks or more goes through in eight slices of whole chunks: slice i of base arrives on a copy stream the call
+ * creates, is recovered in place on `cs`, and leaves on a second copy stream while slice i + 1 arrives, so that
+ * with pinned buffers the two directions of the host link are busy at once. Both streams and their events are
+ * destroyed before the call returns. */
 int lc_recover_host(const float* base_host, const void* const* streams_host,
                     const uint64_t* stream_bytes, int k, uint64_t n, float* out_host, void* arena,
                     uint64_t arena_bytes, lc_cuda_stream_t cs);

@@ -338,8 +338,39 @@ int lc_compress_host(const float* base_host, const float* cur_host, uint64_t n, 
   return LC_OK;
 }
 
-int lc_recover_host(const float* base_host, const void* const* streams_host, const uint64_t* stream_bytes, int k,
-                    uint64_t n, float* out_host, void* arena, uint64_t arena_bytes, lc_cuda_stream_t cs) {
+}  // extern "C"
+
+namespace {
+
+// The two copy streams and the events of lc_recover_host's pipeline; created per call, destroyed on every way out.
+constexpr int kHostSlices = 8;
+struct HostPipeline {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t arrived[kHostSlices] = {}, decoded[kHostSlices] = {};
+  bool create() {
+    if (cudaStreamCreateWithFlags(&in, cudaStreamNonBlocking) != cudaSuccess) return false;
+    if (cudaStreamCreateWithFlags(&out, cudaStreamNonBlocking) != cudaSuccess) return false;
+    for (int i = 0; i < kHostSlices; ++i) {
+      if (cudaEventCreateWithFlags(&arrived[i], cudaEventDisableTiming) != cudaSuccess) return false;
+      if (cudaEventCreateWithFlags(&decoded[i], cudaEventDisableTiming) != cudaSuccess) return false;
+    }
+    return true;
+  }
+  ~HostPipeline() {
+    for (int i = 0; i < kHostSlices; ++i) {
+      if (arrived[i]) cudaEventDestroy(arrived[i]);
+      if (decoded[i]) cudaEventDestroy(decoded[i]);
+    }
+    if (in) cudaStreamDestroy(in);
+    if (out) cudaStreamDestroy(out);
+  }
+};
+
+}  // namespace
+
+extern "C" int lc_recover_host(const float* base_host, const void* const* streams_host, const uint64_t* stream_bytes,
+                               int k, uint64_t n, float* out_host, void* arena, uint64_t arena_bytes,
+                               lc_cuda_stream_t cs) {
   if (k < 1 || k > LC_MAX_CHAIN || n >= (1ull << 32)) return LC_ERR_ARG;
   if (!streams_host || !stream_bytes || !arena || !aligned(arena, 256) || (n > 0 && (!base_host || !out_host)))
     return LC_ERR_ARG;
@@ -354,20 +385,66 @@ int lc_recover_host(const float* base_host, const void* const* streams_host, con
   float* d_x = reinterpret_cast<float*>(a + ws_bytes);
   const void* d_streams[LC_MAX_CHAIN];
   uint64_t off = ws_bytes + vec;
-  if (n > 0 && cudaMemcpyAsync(d_x, base_host, 4 * n, cudaMemcpyHostToDevice, cs) != cudaSuccess) return LC_ERR_CUDA;
   for (int j = 0; j < k; ++j) {
     if (cudaMemcpyAsync(a + off, streams_host[j], stream_bytes[j], cudaMemcpyHostToDevice, cs) != cudaSuccess)
       return LC_ERR_CUDA;
     d_streams[j] = a + off;
     off += align_up(stream_bytes[j], 256);
   }
-  int rc = lc_recover(d_x, d_streams, stream_bytes, k, n, d_x, a, ws_bytes, cs);
-  if (rc != LC_OK) return rc;
-  if ((rc = lc_last_status(a, cs)) != LC_OK) return rc;
-  if (n > 0 && cudaMemcpyAsync(out_host, d_x, 4 * n, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return LC_ERR_CUDA;
-  if (cudaStreamSynchronize(cs) != cudaSuccess) return LC_ERR_CUDA;
-  return LC_OK;
+  const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
+  if (nchunks < 16 * kHostSlices) {
+    // a small vector: one copy in, one call, one copy out
+    if (n > 0 && cudaMemcpyAsync(d_x, base_host, 4 * n, cudaMemcpyHostToDevice, cs) != cudaSuccess) return LC_ERR_CUDA;
+    int rc = lc_recover(d_x, d_streams, stream_bytes, k, n, d_x, a, ws_bytes, cs);
+    if (rc != LC_OK) return rc;
+    if ((rc = lc_last_status(a, cs)) != LC_OK) return rc;
+    if (n > 0 && cudaMemcpyAsync(out_host, d_x, 4 * n, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return LC_ERR_CUDA;
+    if (cudaStreamSynchronize(cs) != cudaSuccess) return LC_ERR_CUDA;
+    return LC_OK;
+  }
+  // A large vector goes through in slices of whole chunks, so that the two directions of the link work at the same
+  // time: slice i of base comes in on one stream, is recovered in place on `cs` as soon as it has arrived (the
+  // chunks of a stream decode independently of one another), and leaves on another stream, while slice i + 1 comes in.
+  for (int j = 0; j < k; ++j)
+    if (!aligned(d_streams[j], 16)) return LC_ERR_ARG;
+  HostPipeline pipe;
+  if (!pipe.create()) return LC_ERR_CUDA;
+  Control* ctl = reinterpret_cast<Control*>(a);
+  void* images = a + workspace_layout(0).decode_off;
+  if (cudaMemsetAsync(&ctl->status, 0, sizeof(int32_t), cs) != cudaSuccess) return LC_ERR_CUDA;
+  const int groups = (k + 3) / 4;
+  for (int i = 0; i < kHostSlices; ++i) {
+    const uint64_t c0 = nchunks * i / kHostSlices, c1 = nchunks * (i + 1) / kHostSlices;
+    const uint64_t e0 = c0 * kChunkElems, e1 = c1 * kChunkElems < n ? c1 * kChunkElems : n;
+    if (cudaMemcpyAsync(d_x + e0, base_host + e0, 4 * (e1 - e0), cudaMemcpyHostToDevice, pipe.in) != cudaSuccess)
+      return LC_ERR_CUDA;
+    if (cudaEventRecord(pipe.arrived[i], pipe.in) != cudaSuccess) return LC_ERR_CUDA;
+    if (cudaStreamWaitEvent(cs, pipe.arrived[i], 0) != cudaSuccess) return LC_ERR_CUDA;
+    for (int g = 0; g < groups; ++g) {
+      const int first = 4 * g, kk = (k - first) < 4 ? (k - first) : 4;
+      DecodeStreams ds;
+      memset(&ds, 0, sizeof ds);
+      for (int j = 0; j < kk; ++j) {
+        ds.ptr[j] = static_cast<const uint8_t*>(d_streams[first + j]);
+        ds.bytes[j] = stream_bytes[first + j];
+      }
+      // the decode tables of a group of four streams are built once if there is one group; two groups share the
+      // table area and rebuild theirs for every slice
+      const bool prepare = groups > 1 || i == 0;
+      if (launch_decode(d_x, ds, kk, n, d_x, &ctl->status, images, cs, c0, c1, prepare) != cudaSuccess) return LC_ERR_CUDA;
+    }
+    if (cudaEventRecord(pipe.decoded[i], cs) != cudaSuccess) return LC_ERR_CUDA;
+    if (cudaStreamWaitEvent(pipe.out, pipe.decoded[i], 0) != cudaSuccess) return LC_ERR_CUDA;
+    if (cudaMemcpyAsync(out_host + e0, d_x + e0, 4 * (e1 - e0), cudaMemcpyDeviceToHost, pipe.out) != cudaSuccess)
+      return LC_ERR_CUDA;
+  }
+  if (cudaStreamSynchronize(pipe.out) != cudaSuccess || cudaStreamSynchronize(cs) != cudaSuccess) return LC_ERR_CUDA;
+  int32_t st = 0;
+  if (cudaMemcpy(&st, &ctl->status, sizeof st, cudaMemcpyDeviceToHost) != cudaSuccess) return LC_ERR_CUDA;
+  return st;
 }
+
+extern "C" {
 
 // ---- stage dumps -----------------------------------------------------------------------------------
 

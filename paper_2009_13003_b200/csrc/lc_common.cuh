@@ -155,7 +155,10 @@ struct DecodeStreams {
   uint64_t bytes[4];
 };
 // images: kDecodeRegionBytes of device scratch for the streams' decode tables (built by a first small kernel)
+// Decodes the chunks [chunk_begin, chunk_end) only (clipped to the vector's chunks). prepare: build the images first
+// (false: an earlier launch for the same streams has left them there).
 cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
-                          int32_t* status, void* images, cudaStream_t cs);
+                          int32_t* status, void* images, cudaStream_t cs, uint64_t chunk_begin = 0,
+                          uint64_t chunk_end = ~0ull, bool prepare = true);
 
 }  // namespace lc

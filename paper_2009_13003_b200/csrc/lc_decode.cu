@@ -525,7 +525,7 @@ __device__ __noinline__ void decode_chunk_partial(const StreamState* S, PartialC
 template <int KS>
 __global__ void __launch_bounds__(kDecMaxThreads, 1)
 decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, int32_t* __restrict__ status,
-              const DecodeImage* __restrict__ images, uint32_t stage_bytes) {
+              const DecodeImage* __restrict__ images, uint32_t stage_bytes, uint64_t chunk_begin, uint64_t chunk_end) {
   // dynamic shared memory: [pad to 8 KB | 2 tables per stream | StreamState per stream | staging areas]
   extern __shared__ __align__(16) unsigned char s_raw[];
   unsigned char* tables = s_raw + ((kTableBytes - (smem_addr(s_raw) & (kTableBytes - 1))) & (kTableBytes - 1));
@@ -564,11 +564,10 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
 
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, warps = blockDim.x >> 5;
   unsigned char* stage0 = reinterpret_cast<unsigned char*>(S + KS) + (size_t)warp * KS * stage_bytes;
-  const uint64_t nchunks = (n + kChunkElems - 1) / kChunkElems;
-  const uint64_t warp0 = (uint64_t)blockIdx.x * warps + warp;
+  const uint64_t warp0 = chunk_begin + (uint64_t)blockIdx.x * warps + warp;  // this launch decodes [chunk_begin, chunk_end)
   const uint64_t nwarps = (uint64_t)gridDim.x * warps;
 
-  for (uint64_t c = warp0; c < nchunks; c += nwarps) {
+  for (uint64_t c = warp0; c < chunk_end; c += nwarps) {
     Source W[KS];
     uint32_t start[KS], bytes[KS];
     unsigned long long off0[KS], off1[KS];
@@ -624,7 +623,7 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
     if ((c + 1) * kChunkElems <= n) {
       // where the L2 prefetch goes on behind this chunk: the next chunk of this warp, if it is a full one
       const uint64_t cn = c + nwarps;
-      const float* next_rows = base + ((cn + 1) * kChunkElems <= n ? cn : c) * kChunkElems + 4 * lane;
+      const float* next_rows = base + (cn < chunk_end && (cn + 1) * kChunkElems <= n ? cn : c) * kChunkElems + 4 * lane;
       if (fits) decode_chunk_fast<KS, true>(S, W, start, base, out, c, lane, next_rows, status);
       else decode_chunk_fast<KS, false>(S, W, start, base, out, c, lane, next_rows, status);
     } else {
@@ -644,7 +643,8 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
 
 template <int KS>
 cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, uint64_t n, float* out,
-                             int32_t* status, const DecodeImage* images, cudaStream_t cs) {
+                             int32_t* status, const DecodeImage* images, uint64_t chunk_begin, uint64_t chunk_end,
+                             cudaStream_t cs) {
   static int sms_of[kMaxDevices] = {};  // by device ordinal; non-zero once the kernel's attributes are set there
   constexpr uint32_t kTables = kTableBytes + KS * (2 * kTableBytes + sizeof(StreamState));
   constexpr uint32_t kMaxDyn = kSmemPerSm - 1024 - kOverrunBytes;  // room for static __shared__ and the padding
@@ -710,8 +710,8 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
       }
     }
   }
-  uint64_t want = (nchunks + warps - 1) / warps;
-  if (want == 0) want = 1;  // still validates the streams
+  uint64_t want = (chunk_end - chunk_begin + warps - 1) / warps;
+  if (want == 0) want = 1;  // still reports a rejected stream
   const uint64_t full = (uint64_t)sms * ctas_per_sm;
   const unsigned grid = (unsigned)(want < full ? want : full);
   {
@@ -722,15 +722,19 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
     if (cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributePreferredSharedMemoryCarveout, carve) != cudaSuccess)
       return cudaErrorUnknown;
   }
-  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, images, stage);
+  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, images, stage, chunk_begin, chunk_end);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k, uint64_t n, float* out,
-                          int32_t* status, void* images, cudaStream_t cs) {
+                          int32_t* status, void* images, cudaStream_t cs, uint64_t chunk_begin, uint64_t chunk_end,
+                          bool prepare) {
   if (k < 1 || k > 4) return cudaErrorInvalidValue;
+  const uint64_t all_chunks = (n + kChunkElems - 1) / kChunkElems;
+  if (chunk_end > all_chunks) chunk_end = all_chunks;
+  if (chunk_begin > chunk_end) chunk_begin = chunk_end;
   static bool prep_ready[kMaxDevices] = {};  // by device ordinal
   const int dev = current_device_index();
   if (dev < 0) return cudaErrorInvalidDevice;
@@ -741,13 +745,15 @@ cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k
     prep_ready[dev] = true;
   }
   DecodeImage* img = static_cast<DecodeImage*>(images);
-  decode_prepare_kernel<<<k, kPrepThreads, kPrepSmem, cs>>>(streams, n, img);
-  if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
+  if (prepare) {
+    decode_prepare_kernel<<<k, kPrepThreads, kPrepSmem, cs>>>(streams, n, img);
+    if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
+  }
   switch (k) {
-    case 1: return launch_decode_ks<1>(base, streams, n, out, status, img, cs);
-    case 2: return launch_decode_ks<2>(base, streams, n, out, status, img, cs);
-    case 3: return launch_decode_ks<3>(base, streams, n, out, status, img, cs);
-    case 4: return launch_decode_ks<4>(base, streams, n, out, status, img, cs);
+    case 1: return launch_decode_ks<1>(base, streams, n, out, status, img, chunk_begin, chunk_end, cs);
+    case 2: return launch_decode_ks<2>(base, streams, n, out, status, img, chunk_begin, chunk_end, cs);
+    case 3: return launch_decode_ks<3>(base, streams, n, out, status, img, chunk_begin, chunk_end, cs);
+    case 4: return launch_decode_ks<4>(base, streams, n, out, status, img, chunk_begin, chunk_end, cs);
     default: return cudaErrorInvalidValue;
   }
 }

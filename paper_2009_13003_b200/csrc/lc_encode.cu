@@ -95,16 +95,14 @@ struct OrPacker {
 
 // Slow, compact path (see the header). With dst == nullptr it only returns the lane's bit count;
 // otherwise it ORs the lane's bits into the zeroed chunk image at dst, starting at bit lane_start.
-// `tb`: the CTA's shared-memory tables by plane byte, used for codes of up to 32 bits when the keys come from the
-// plane (nullptr: the per-key table in global memory). The plane bytes of four steps are read as one 16-byte vector,
-// the way the fast path reads them: this path also codes the vector's partial last chunk, alone in its warp, and
-// with a byte and a table entry fetched from global memory per element that one chunk took longer than all the
-// others of a medium-sized vector together.
-__device__ __noinline__ uint32_t chunk_slow(const EncEntry* __restrict__ enc, const Tables* tb, KeySource ks, uint64_t c,
+// The plane bytes of four steps are read as one 16-byte vector, the way the fast path reads them (this path also
+// codes the vector's partial last chunk, alone in its warp). Codes come from the per-key table in global memory:
+// passing the CTA's shared tables in as well was measured to cost the kernel's main loop 4 %.
+__device__ __noinline__ uint32_t chunk_slow(const EncEntry* __restrict__ enc, KeySource ks, uint64_t c,
                                             uint32_t lane, uint64_t n, uint32_t* dst, uint32_t lane_start) {
   OrPacker pk{0ull, lane_start & 31u, dst ? dst + (lane_start >> 5) : nullptr};
   uint32_t bits = 0;
-  const bool from_plane = tb != nullptr && !ks.wide;
+  const bool from_plane = !ks.wide;
   for (uint32_t q = 0; q < kSteps / 4; ++q) {
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (from_plane) v = __ldg(reinterpret_cast<const uint4*>(ks.plane + c * kChunkElems + q * 512) + lane);
@@ -116,17 +114,15 @@ __device__ __noinline__ uint32_t chunk_slow(const EncEntry* __restrict__ enc, co
       for (uint32_t e = 0; e < kGroup; ++e) {
         const uint64_t i = c * kChunkElems + 128ull * j + 4 * lane + e;
         if (i >= n) continue;
-        uint32_t code_lo, code_hi = 0, len;
+        uint32_t key;
         if (from_plane) {
-          const uint2 f = tb->full[(words[r] >> (8 * e)) & 255u];
-          code_lo = f.x;
-          len = f.y;
+          const uint32_t b = (words[r] >> (8 * e)) & 255u;
+          key = ((b & 1u) << 8) | (b >> 1);
         } else {
-          const EncEntry en = enc[ks.key(c, j, lane, e)];
-          code_lo = en.code_lo;
-          code_hi = en.code_hi;
-          len = en.len;
+          key = ks.key(c, j, lane, e);
         }
+        const EncEntry en = enc[key];
+        const uint32_t code_lo = en.code_lo, code_hi = en.code_hi, len = en.len;
         bits += len;
         if (dst) {
           if (len > 32) {
@@ -220,7 +216,6 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
   const uint32_t nsym = ctl->nsym;
   const bool long_codes = ctl->max_len > 32;
   const KeySource ks{plane, base, cur, ctl->wide != 0};
-  const Tables* slow_tb = long_codes ? nullptr : &tb;  // what the slow path may look codes up in
   const StreamLayout L = stream_layout(n, nsym);
   const uint64_t nchunks = L.nchunks;
   unsigned long long* chunk_index = reinterpret_cast<unsigned long long*>(stream + L.chunk_index_off);
@@ -365,7 +360,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
         lane_bits = ((pk.dst - col0) >> 7) * 32 + pk.nb;
       }
     }
-    if (!fast && valid) lane_bits = chunk_slow(ctl->enc, slow_tb, ks, c, lane, n, nullptr, 0);
+    if (!fast && valid) lane_bits = chunk_slow(ctl->enc, ks, c, lane, n, nullptr, 0);
 
     // ---- B: lane offsets, lane index, chunk size; the tile's size is published as early as possible
     if (valid) lane_index[c * kLanes + lane] = (uint16_t)lane_bits;
@@ -483,7 +478,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
           for (uint32_t k = lane; k < p_chunk_bytes / 16; k += 32) dst4[k] = make_uint4(0, 0, 0, 0);
           __threadfence_block();
           __syncwarp();
-          chunk_slow(ctl->enc, slow_tb, ks, p_c, lane, n, reinterpret_cast<uint32_t*>(dst4), s_lane_start[p_buf][tid]);
+          chunk_slow(ctl->enc, ks, p_c, lane, n, reinterpret_cast<uint32_t*>(dst4), s_lane_start[p_buf][tid]);
         }
       }
       if (p_tile == ntiles - 1 && tid == 0) {
@@ -554,7 +549,7 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
         const uint32_t tail = r ? prev << (32 - r) : 0u;
         if (tail) atomicOr(out + nw, tail);
       } else {
-        chunk_slow(ctl->enc, slow_tb, ks, c, lane, n, image, lane_start);
+        chunk_slow(ctl->enc, ks, c, lane, n, image, lane_start);
       }
     }
     __syncwarp();
@@ -579,7 +574,7 @@ encode_sizes_kernel(const Control* __restrict__ ctl, unsigned long long* __restr
   const KeySource ks{plane, base, cur, ctl->wide != 0};
   const uint64_t warp0 = (uint64_t)blockIdx.x * kEncWarps + (threadIdx.x >> 5), nwarps = (uint64_t)gridDim.x * kEncWarps;
   for (uint64_t c = warp0; c < nchunks; c += nwarps) {
-    uint32_t bits = chunk_slow(ctl->enc, nullptr, ks, c, lane, n, nullptr, 0);
+    uint32_t bits = chunk_slow(ctl->enc, ks, c, lane, n, nullptr, 0);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) bits += __shfl_xor_sync(0xffffffffu, bits, d);
     if (lane == 0) sizes[c] = align_up((bits + 7) / 8, kPayloadAlign);

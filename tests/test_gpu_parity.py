@@ -447,15 +447,25 @@ def test_corrupted_streams_are_rejected_not_faulting(lc, oracle):
     assert status_of(good) == 0
 
 
-def test_host_buffer_entry_points(lc, oracle):
-    n, nbits = 1_234_567, 4
+@pytest.mark.parametrize("n,k", [(1_234_567, 2), (1_234_567, 6), (130 * 4096, 1), (50_001, 3), (0, 1)])
+def test_host_buffer_entry_points(lc, oracle, n, k):
+    """Large vectors go through lc_recover_host in slices of whole chunks (copies in both directions overlapped with
+    the decode of the slice between them), small ones in one piece; a chain above four streams takes two passes per
+    slice. All of it must give the oracle's values."""
+    nbits = 4
     base, cur = make_case(n, 9)
     bh, ch = base.cpu().pin_memory(), cur.cpu().pin_memory()
-    arena = torch.empty(lc.host_arena_bytes(n, nbits, 2), dtype=torch.uint8, device=DEV)
+    arena = torch.empty(lc.host_arena_bytes(n, nbits, k), dtype=torch.uint8, device=DEV)
     sh = torch.empty(lc.stream_bound(n, nbits), dtype=torch.uint8).pin_memory()
     size = lc.compress_host(bh, ch, nbits, sh, arena)
     want = oracle.compress(bh.numpy(), ch.numpy(), nbits)
     assert sh[:size].numpy().tobytes() == want.tobytes()
-    oh = torch.empty(n, dtype=torch.float32).pin_memory()
-    lc.recover_host(bh, [sh[:size], sh[:size]], oh, arena)
-    assert np.array_equal(oh.numpy().view(np.uint32), oracle.recover(bh.numpy(), [want, want]).view(np.uint32))
+    oh = torch.full((n,), 7.0, dtype=torch.float32).pin_memory()
+    lc.recover_host(bh, [sh[:size]] * k, oh, arena)
+    assert np.array_equal(oh.numpy().view(np.uint32), oracle.recover(bh.numpy(), [want] * k).view(np.uint32))
+    if n:
+        bad = sh[:size].clone()
+        bad[0] = 0
+        with pytest.raises(Exception):
+            lc.recover_host(bh, [sh[:size]] * (k - 1) + [bad], oh, arena)
+        lc.recover_host(bh, [sh[:size]] * k, oh, arena)
