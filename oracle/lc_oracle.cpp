@@ -17,7 +17,9 @@
 // lco_recover of lco_compress, lco_compress_chunks to slices of lco_compress's stream, the threaded
 // timing mode to the single-threaded bytes, lco_merge to the idempotence of quantization over a zero
 // base (the merged stream of one stream is that stream) and to Algorithm 1 step 7 applied to the
-// recovered state.
+// recovered state. The length cache of Section 3.2 (lco_cached_lengths, lco_compress_cached) is pinned by hand-worked
+// rows and assignments, by byte equality with the plain stream on an empty cache, and by a cached stream
+// recovering the plain stream's state with more payload bits than the plain stream's optimal code.
 // Parity unpinned: the whole-pipeline result on the paper's own training deltas (its figures carry
 // the only values and they are not available); only the loose size ranges of Section 4.3 apply.
 
@@ -196,6 +198,7 @@ struct Table {
   int max_len = 0;
   int fixed = 0;   // 1: fixed-width codes (format section 1.5) instead of the Huffman code
   int shared = 0;  // 1: the table was built from a larger vector than the stream codes (format section 1.6)
+  int cached = 0;  // 1: the code lengths were taken from a length cache (format section 1.7)
   int key[512] = {};
   int len[512] = {};
   float rep[512] = {};
@@ -204,7 +207,47 @@ struct Table {
 };
 
 // Steps of Sections 3.1.1-3.1.2 that turn bucket statistics into the symbol table.
-int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selection* sel_out, int fixed = 0) {
+// Section 3.2, "Huffman Code Table Caching": the code table of an earlier snapshot with the same number of buckets
+// is used again, the buckets only being sorted by their numbers of entries. The cache (format section 1.7) has one
+// row of 512 bytes per number u of used symbols, row u - 1: the u code lengths in ascending order, valid if its
+// first byte is not 0. A valid row gives the r-th most frequent used symbol (ties: smaller id first) the r-th
+// length, provided the payload then stays within n * nbits bits (the stream bound); otherwise the Huffman lengths
+// are built and written to the row. Returns 1 if the lengths came from the cache.
+constexpr int kCacheRowBytes = 512;
+int cached_lengths(const uint64_t* count, int nsym, int nbits, uint64_t n, uint8_t* cache, int* len /*[nsym]*/) {
+  std::vector<int> used;
+  for (int j = 0; j < nsym; ++j)
+    if (count[j] > 0) used.push_back(j);
+  const int u = static_cast<int>(used.size());
+  if (u < 2) {
+    for (int j = 0; j < nsym; ++j) len[j] = 0;
+    return 0;
+  }
+  uint8_t* row = cache + static_cast<size_t>(kCacheRowBytes) * (u - 1);
+  if (row[0] != 0) {
+    std::stable_sort(used.begin(), used.end(), [&](int a, int b) {
+      if (count[a] != count[b]) return count[a] > count[b];
+      return a < b;
+    });
+    unsigned __int128 bits = 0;
+    for (int r = 0; r < u; ++r) bits += static_cast<unsigned __int128>(count[used[r]]) * row[r];
+    if (bits <= static_cast<unsigned __int128>(n) * static_cast<unsigned>(nbits)) {
+      for (int j = 0; j < nsym; ++j) len[j] = 0;
+      for (int r = 0; r < u; ++r) len[used[r]] = row[r];
+      return 1;
+    }
+  }
+  huffman_lengths(count, nsym, len);
+  std::vector<int> sorted;
+  for (int j = 0; j < nsym; ++j)
+    if (count[j] > 0) sorted.push_back(len[j]);
+  std::sort(sorted.begin(), sorted.end());
+  for (int r = 0; r < kCacheRowBytes; ++r) row[r] = r < u ? static_cast<uint8_t>(sorted[r]) : 0;
+  return 0;
+}
+
+int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selection* sel_out, int fixed = 0,
+                uint8_t* cache = nullptr) {
   for (int s = 0; s <= 1; ++s)
     if (buckets[256 * s + 255].count > 0) return LCO_ERR_NONFINITE;
   const Selection sel = priority_promotion(buckets, nbits);
@@ -232,7 +275,8 @@ int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selectio
       t->code[j] = static_cast<uint64_t>(j);
     }
   } else {
-    huffman_lengths(t->count, t->nsym, t->len);
+    if (cache) t->cached = cached_lengths(t->count, t->nsym, nbits, n, cache, t->len);
+    else huffman_lengths(t->count, t->nsym, t->len);
     canonical_codes(t->len, t->nsym, t->code);
   }
   for (int j = 0; j < t->nsym; ++j) t->max_len = std::max(t->max_len, t->len[j]);
@@ -334,8 +378,10 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   if (!(s[0] == 'L' && s[1] == 'C' && s[2] == 'C' && s[3] == '1')) return LCO_ERR_FORMAT;
   if (get_le(s + 4, 2) != 1) return LCO_ERR_FORMAT;
   const int nbits = static_cast<int>(s[6]);
-  if (nbits < 1 || nbits > 9 || s[7] > 3) return LCO_ERR_FORMAT;
-  const int fixed = static_cast<int>(s[7] & 1), shared = static_cast<int>(s[7] >> 1);
+  if (nbits < 1 || nbits > 9 || s[7] > 7) return LCO_ERR_FORMAT;
+  const int fixed = static_cast<int>(s[7] & 1), shared = static_cast<int>((s[7] >> 1) & 1);
+  const int cached = static_cast<int>((s[7] >> 2) & 1);
+  if (cached && (fixed || shared)) return LCO_ERR_FORMAT;
   const uint64_t n = get_le(s + 8, 8);
   const uint64_t nsym = get_le(s + 16, 4);
   const uint64_t max_len = get_le(s + 20, 4);
@@ -377,6 +423,7 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   p.table.max_len = seen_max;
   p.table.fixed = fixed;
   p.table.shared = shared;
+  p.table.cached = cached;
   if (fixed) {
     int width = 0;
     while ((1ull << width) < nsym) width += 1;
@@ -513,7 +560,7 @@ void write_header_and_table(uint8_t* stream, const Table& t, uint64_t n, int nbi
   h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
   put_le(h + 4, 1, 2);
   h[6] = static_cast<uint8_t>(nbits);
-  h[7] = static_cast<uint8_t>(t.fixed | (t.shared << 1));
+  h[7] = static_cast<uint8_t>(t.fixed | (t.shared << 1) | (t.cached << 2));
   put_le(h + 8, n, 8);
   put_le(h + 16, static_cast<uint64_t>(t.nsym), 4);
   put_le(h + 20, static_cast<uint64_t>(t.max_len), 4);
@@ -624,15 +671,16 @@ uint64_t lco_stream_bound(uint64_t n, int nbits) { return stream_bound(n, nbits)
 // Full compress pass: Algorithm 1 steps 4-6. Writes the stream, returns its size through *out_bytes.
 // `fixed`: 0 for the Huffman code (Section 3.1.2), 1 for fixed-width bucket indices (the size model of
 // Section 3.1.1 and the "E" / "E+P" stages of Section 4.3's size breakdown).
-int lco_compress_mode(const float* base, const float* cur, uint64_t n, int nbits, int fixed, uint8_t* stream,
-                      uint64_t capacity, uint64_t* out_bytes) {
-  if (nbits < 1 || nbits > 9 || fixed < 0 || fixed > 1 || n >= (1ull << 32)) return LCO_ERR_ARG;
+// `cache`: null, or the length cache of Section 3.2's "Huffman Code Table Caching" (read and updated).
+static int compress_body(const float* base, const float* cur, uint64_t n, int nbits, int fixed, uint8_t* cache,
+                         uint8_t* stream, uint64_t capacity, uint64_t* out_bytes) {
+  if (nbits < 1 || nbits > 9 || fixed < 0 || fixed > 1 || n >= (1ull << 32) || (cache && fixed)) return LCO_ERR_ARG;
   if (capacity < stream_bound(n, nbits)) return LCO_ERR_CAPACITY;
   std::vector<Bucket> buckets(512);
   delta_buckets(base, cur, n, buckets.data());
   Table t;
   Selection sel;
-  const int rc = build_table(buckets.data(), n, nbits, &t, &sel, fixed);
+  const int rc = build_table(buckets.data(), n, nbits, &t, &sel, fixed, cache);
   if (rc != LCO_OK) return rc;
 
   const Layout L = layout_for(n, t.nsym);
@@ -655,6 +703,23 @@ int lco_compress_mode(const float* base, const float* cur, uint64_t n, int nbits
   write_header_and_table(stream, t, n, nbits, L, payload_bits, payload_bytes);
   *out_bytes = L.payload_off + payload_bytes;
   return LCO_OK;
+}
+
+int lco_compress_mode(const float* base, const float* cur, uint64_t n, int nbits, int fixed, uint8_t* stream,
+                      uint64_t capacity, uint64_t* out_bytes) {
+  return compress_body(base, cur, n, nbits, fixed, nullptr, stream, capacity, out_bytes);
+}
+
+// Compress pass with the length cache of Section 3.2 ("Huffman Code Table Caching"); cache: 512 rows of 512 bytes.
+int lco_compress_cached(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* cache, uint8_t* stream,
+                        uint64_t capacity, uint64_t* out_bytes) {
+  if (!cache) return LCO_ERR_ARG;
+  return compress_body(base, cur, n, nbits, 0, cache, stream, capacity, out_bytes);
+}
+
+// The caching step alone: code lengths of `nsym` symbols with the given counts (n = their sum). Returns 1 on a hit.
+int lco_cached_lengths(const uint64_t* count, int nsym, int nbits, uint64_t n, uint8_t* cache, int* len) {
+  return cached_lengths(count, nsym, nbits, n, cache, len);
 }
 
 int lco_compress(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* stream,

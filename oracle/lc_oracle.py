@@ -38,6 +38,8 @@ def lib():
         L.lco_table_mode.argtypes = [vp, vp, u64, i32, i32, vp, vp, vp, vp, vp]
         L.lco_compress_mode.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_mode_mt.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64), i32]
+        L.lco_compress_cached.argtypes = [vp, vp, u64, i32, vp, vp, u64, C.POINTER(u64)]
+        L.lco_cached_lengths.argtypes = [vp, i32, i32, u64, vp, vp]
         L.lco_compress_shard.argtypes = [vp, vp, u64, u64, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_mt.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), i32]
@@ -135,6 +137,37 @@ def compress(base, cur, nbits, threads=None, fixed=False):
     if rc < 0:
         raise OracleError(rc)
     return buf[: out.value].copy()
+
+
+CACHE_BYTES = 512 * 512
+
+
+def new_cache():
+    """An empty length cache (Section 3.2, "Huffman Code Table Caching"): 512 rows of 512 bytes, all zero."""
+    return np.zeros(CACHE_BYTES, np.uint8)
+
+
+def compress_cached(base, cur, nbits, cache):
+    """Compress pass that reads and updates the length cache ``cache`` (uint8[CACHE_BYTES], changed in place)."""
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    assert cache.dtype == np.uint8 and cache.size == CACHE_BYTES and cache.flags.c_contiguous
+    cap = stream_bound(base.size, nbits)
+    buf = np.zeros(cap, np.uint8)
+    out = C.c_uint64(0)
+    rc = lib().lco_compress_cached(pb, pc, base.size, nbits, cache.ctypes.data, buf.ctypes.data, cap, C.byref(out))
+    if rc < 0:
+        raise OracleError(rc)
+    return buf[: out.value].copy()
+
+
+def cached_lengths(count, nbits, cache):
+    """The caching step alone: (hit, code lengths) for symbols with the given counts; ``cache`` changed in place."""
+    count = np.ascontiguousarray(count, dtype=np.uint64)
+    ln = np.zeros(count.size, np.int32)
+    hit = lib().lco_cached_lengths(count.ctypes.data, count.size, nbits, int(count.sum()), cache.ctypes.data,
+                                   ln.ctypes.data)
+    return bool(hit), ln
 
 
 def compress_shard(base, cur, lo, hi, nbits):

@@ -61,6 +61,12 @@ MUTATIONS = [
     ("shard codes from the vector's first element", "payload_bytes += encode_chunk(base + lo, cur + lo, n, t, sel, c,", "payload_bytes += encode_chunk(base, cur, n, t, sel, c,"),
     ("shard's table built from the shard alone", "delta_buckets(base, cur, n_total, buckets.data());\n  Table t;\n  Selection sel;\n  const int rc = build_table(buckets.data(), n_total, nbits, &t, &sel);\n  if (rc != LCO_OK) return rc;\n  t.shared = 1;",
      "delta_buckets(base + lo, cur + lo, hi - lo, buckets.data());\n  Table t;\n  Selection sel;\n  const int rc = build_table(buckets.data(), hi - lo, nbits, &t, &sel);\n  if (rc != LCO_OK) return rc;\n  t.shared = 1;"),
+    ("cache: least frequent symbol gets the shortest length", "if (count[a] != count[b]) return count[a] > count[b];", "if (count[a] != count[b]) return count[a] < count[b];"),
+    ("cache: size bound not checked", "if (bits <= static_cast<unsigned __int128>(n) * static_cast<unsigned>(nbits)) {", "if (bits > 0) {"),
+    ("cache: row chosen by the table size", "uint8_t* row = cache + static_cast<size_t>(kCacheRowBytes) * (u - 1);", "uint8_t* row = cache + static_cast<size_t>(kCacheRowBytes) * (nsym - 1);"),
+    ("cache: row stored unsorted", "std::sort(sorted.begin(), sorted.end());", ""),
+    ("cache: a hit is coded with the Huffman lengths", "if (cache) t->cached = cached_lengths(t->count, t->nsym, nbits, n, cache, t->len);\n    else huffman_lengths(t->count, t->nsym, t->len);",
+     "if (cache) { std::vector<int> tmp(512); t->cached = cached_lengths(t->count, t->nsym, nbits, n, cache, tmp.data()); }\n    huffman_lengths(t->count, t->nsym, t->len);"),
     ("size model uses floor log", "while ((1ull << width) < k) width += 1;", "while ((2ull << width) <= k) width += 1;"),
 ]
 
@@ -91,6 +97,8 @@ class _Oracle:
         L.lco_midrange.restype = C.c_float
         L.lco_compress_mode.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_shard.argtypes = [vp, vp, u64, u64, u64, i32, vp, u64, C.POINTER(u64)]
+        L.lco_compress_cached.argtypes = [vp, vp, u64, i32, vp, vp, u64, C.POINTER(u64)]
+        L.lco_cached_lengths.argtypes = [vp, i32, i32, u64, vp, vp]
         L.lco_apply_quantized.argtypes = [vp, vp, u64, i32, vp]
         L.lco_compress_chunks.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
         L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
@@ -104,6 +112,20 @@ class _Oracle:
         out = C.c_uint64(0)
         assert self.L.lco_compress_mode(base.ctypes.data, cur.ctypes.data, base.size, nbits, 1, buf.ctypes.data, cap,
                                         C.byref(out)) == 0
+        return buf[: out.value].copy()
+
+    def cached_lengths(self, counts, nbits, cache):
+        c = np.asarray(counts, np.uint64)
+        ln = np.zeros(c.size, np.int32)
+        hit = self.L.lco_cached_lengths(c.ctypes.data, c.size, nbits, int(c.sum()), cache.ctypes.data, ln.ctypes.data)
+        return bool(hit), ln.tolist()
+
+    def compress_cached(self, base, cur, nbits, cache):
+        cap = int(self.L.lco_stream_bound(base.size, nbits))
+        buf = np.zeros(cap + 64, np.uint8)
+        out = C.c_uint64(0)
+        assert self.L.lco_compress_cached(base.ctypes.data, cur.ctypes.data, base.size, nbits, cache.ctypes.data,
+                                          buf.ctypes.data, cap, C.byref(out)) == 0
         return buf[: out.value].copy()
 
     def compress_shard(self, base, cur, lo, hi, nbits):
@@ -297,6 +319,37 @@ def _pins_hold(o):
         whole2 = o.recover(base, [o.compress(base, d2, 2)])
         s2b = o.compress_shard(base, d2, 3000, n, 2)
         if not np.array_equal(o.recover(base[3000:], [s2b]).view(np.uint32), whole2[3000:].view(np.uint32)):
+            return False
+        # code-table caching: hand-worked rows (see test_cached_lengths_hand_worked), then a cached stream
+        cache = np.zeros(512 * 512, np.uint8)
+        rows = cache.reshape(512, 512)
+        if o.cached_lengths([1, 8, 2, 4, 1], 3, cache) != (False, [4, 1, 3, 2, 4]) or rows[4, :6].tolist() != [1, 2, 3, 4, 4, 0]:
+            return False
+        if o.cached_lengths([3, 5, 4, 2, 6], 3, cache) != (True, [4, 2, 3, 4, 1]):
+            return False
+        if o.cached_lengths([9, 0, 7, 1, 1, 2], 3, cache) != (True, [1, 0, 2, 4, 4, 3]):
+            return False
+        o.cached_lengths([128, 64, 32, 16, 8, 4, 2, 1], 3, cache)
+        if o.cached_lengths([10] * 8, 3, cache) != (False, [3] * 8) or rows[7, :9].tolist() != [3] * 8 + [0]:
+            return False
+        cache[:] = 0
+        if o.compress_cached(base, cur, 3, cache).tobytes() != s.tobytes():
+            return False
+        # a Gaussian snapshot fills the row of 8 used symbols with a flatter length list; the Laplace snapshot that
+        # follows is then coded with those lengths (more bits than its own Huffman code, same symbols and state)
+        cache[:] = 0
+        cur_g = (base + rng.normal(0, 1e-3, n).astype(np.float32)).astype(np.float32)
+        o.compress_cached(base, cur_g, 3, cache)
+        sc = o.compress_cached(base, cur, 3, cache)
+        nsb = int(np.frombuffer(sc[16:20].tobytes(), "<u4")[0])
+        tab = np.frombuffer(sc[64:64 + 16 * nsb].tobytes(), dtype=[("key", "<u2"), ("len", "u1"), ("pad", "u1"), ("rep", "<u4"), ("count", "<u8")])
+        used = int(np.count_nonzero(tab["count"]))
+        order = sorted(range(nsb), key=lambda j: (-int(tab["count"][j]), j))[:used]
+        if sc[7] != 4 or [int(tab["len"][j]) for j in order] != rows[used - 1, :used].tolist():
+            return False
+        if int(np.frombuffer(sc[40:48].tobytes(), "<u8")[0]) <= int(np.frombuffer(s[40:48].tobytes(), "<u8")[0]):
+            return False
+        if not np.array_equal(o.recover(base, [sc]).view(np.uint32), once.view(np.uint32)):
             return False
         # the threaded timing mode writes the same bytes and states
         if o.compress_mt(base, cur, 3, 3).tobytes() != s.tobytes():

@@ -709,3 +709,76 @@ def test_shards_code_with_the_whole_vectors_table(oracle):
         bad[7] = 0
         with pytest.raises(oracle.OracleError):
             oracle.recover(base[:4096], [bad])
+
+
+# ---- Section 3.2, "Huffman Code Table Caching" (format section 1.7) ------------------------------------------
+
+
+def test_cached_lengths_hand_worked(oracle):
+    cache = oracle.new_cache()
+    # first snapshot: five used symbols, nothing cached -> the Huffman lengths, and their sorted list in row 4.
+    # The counts are given out of order so that the stored row shows the sort.
+    hit, ln = oracle.cached_lengths([1, 8, 2, 4, 1], 3, cache)
+    assert not hit and ln.tolist() == [4, 1, 3, 2, 4]
+    rows = cache.reshape(512, 512)
+    assert rows[4, :6].tolist() == [1, 2, 3, 4, 4, 0] and not rows[:4].any() and not rows[5:].any() and not rows[4, 5:].any()
+    # second snapshot, again five used symbols: the cached lengths go to the symbols in the order of their counts,
+    # most frequent first. 6+10+12+12+8 = 48 bits <= 20 elements * 3 bits, so the row is used, although the
+    # Huffman code of these counts (lengths 3,2,2,3,2) takes 45.
+    hit, ln = oracle.cached_lengths([3, 5, 4, 2, 6], 3, cache)
+    assert hit and ln.tolist() == [4, 2, 3, 4, 1]
+    assert sum(c * int(l) for c, l in zip([3, 5, 4, 2, 6], ln)) == 48
+    assert sum(c * int(l) for c, l in zip([3, 5, 4, 2, 6], oracle.huffman([3, 5, 4, 2, 6])[0])) == 45
+    assert rows[4, :6].tolist() == [1, 2, 3, 4, 4, 0]  # a hit leaves the row alone
+    # equal counts: the smaller symbol id takes the shorter length
+    hit, ln = oracle.cached_lengths([5, 5, 5, 5, 2], 3, cache)
+    assert hit and ln.tolist() == [1, 2, 3, 4, 4]
+    # an unused symbol in between: the row is chosen by the number of USED symbols and the symbol keeps length 0
+    hit, ln = oracle.cached_lengths([9, 0, 7, 1, 1, 2], 3, cache)
+    assert hit and ln.tolist() == [1, 0, 2, 4, 4, 3]
+    # a row that would break the size bound is rebuilt: eight symbols cached from a skewed snapshot, then a
+    # uniform one: 10 * (1+2+3+4+5+6+7+7) = 350 bits > 80 * 3
+    hit, ln = oracle.cached_lengths([128, 64, 32, 16, 8, 4, 2, 1], 3, cache)
+    assert not hit and ln.tolist() == [1, 2, 3, 4, 5, 6, 7, 7] and rows[7, :9].tolist() == [1, 2, 3, 4, 5, 6, 7, 7, 0]
+    hit, ln = oracle.cached_lengths([10] * 8, 3, cache)
+    assert not hit and ln.tolist() == [3] * 8 and rows[7, :9].tolist() == [3] * 8 + [0]
+    # fewer than two used symbols: no code, cache untouched
+    before = cache.copy()
+    hit, ln = oracle.cached_lengths([0, 7, 0], 2, cache)
+    assert not hit and ln.tolist() == [0, 0, 0] and np.array_equal(cache, before)
+
+
+def test_cached_stream_properties(oracle):
+    rng = np.random.default_rng(123)
+    n, nbits = 3 * 4096 + 500, 3
+    base, cur2 = _random_case(rng, n)  # Laplace deltas: a steep length list
+    cur1 = (base + rng.normal(0, 1e-3, n).astype(np.float32)).astype(np.float32)  # Gaussian: same bucket count, flatter
+    cache = oracle.new_cache()
+    # nothing cached yet: the plain stream, byte for byte, and the row of its used-symbol count gets its lengths
+    s1 = oracle.compress_cached(base, cur1, nbits, cache)
+    assert s1.tobytes() == oracle.compress(base, cur1, nbits).tobytes()
+    p1 = _parse(s1)
+    u = int(np.count_nonzero(p1["tab"]["count"]))
+    assert u == 8
+    rows = cache.reshape(512, 512)
+    assert rows[u - 1, :u].tolist() == sorted(p1["tab"]["len"].tolist()) and rows.sum() == rows[u - 1, :u].sum()
+    # next snapshot: same number of used symbols -> the cached lengths, handed out by count
+    s2 = oracle.compress_cached(base, cur2, nbits, cache)
+    plain2 = oracle.compress(base, cur2, nbits)
+    p2, q2 = _parse(s2), _parse(plain2)
+    assert p2["flags"] == 4 and q2["flags"] == 0
+    for f in ("key", "rep", "count"):
+        assert np.array_equal(p2["tab"][f], q2["tab"][f])
+    order = sorted(range(p2["nsym"]), key=lambda j: (-int(p2["tab"]["count"][j]), j))
+    assert [int(p2["tab"]["len"][j]) for j in order] == rows[u - 1, :u].tolist()
+    assert p2["payload_bits"] == int(np.sum(p2["tab"]["count"] * p2["tab"]["len"].astype(np.uint64)))
+    assert q2["payload_bits"] < p2["payload_bits"] <= n * nbits  # not this snapshot's optimal code, within the bound
+    assert sorted(q2["tab"]["len"].tolist()) != rows[u - 1, :u].tolist()
+    # the stream is an ordinary stream: same symbols, same recovered state as the plain one
+    assert np.array_equal(oracle.decode_symbols(s2, n), oracle.symbols(base, cur2, nbits))
+    assert np.array_equal(oracle.recover(base, [s2]).view(np.uint32), oracle.recover(base, [plain2]).view(np.uint32))
+    # the cached-lengths flag goes with neither fixed-width codes nor shards
+    bad = s2.copy()
+    bad[7] = 5
+    with pytest.raises(oracle.OracleError):
+        oracle.recover(base, [bad])
