@@ -415,7 +415,7 @@ def test_reader_rejects_corruption(oracle):
     expect(setb(0, ord("X")), oracle.ERR_FORMAT)     # magic
     expect(setb(4, 2), oracle.ERR_FORMAT)            # version
     expect(setb(6, 10), oracle.ERR_FORMAT)           # nbits
-    expect(setb(7, 4), oracle.ERR_FORMAT)            # flags
+    expect(setb(7, 8), oracle.ERR_FORMAT)            # flags
     expect(setb(16, 200), oracle.ERR_FORMAT)         # nsym > 2^nbits
     expect(setb(24, 1), oracle.ERR_FORMAT)           # chunk_elems
     expect(setb(64 + 16 + 2, 1), oracle.ERR_FORMAT)  # a code length changed: Kraft / payload_bits
