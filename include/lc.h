@@ -57,6 +57,7 @@ typedef struct lc_info {
   int32_t valid;           /* 1 if magic, version and constants are those of format version 1 */
   uint32_t fixed_width;    /* 1 if the stream carries fixed-width codes (format section 1.5) */
   uint32_t shard;          /* 1 if the stream is a shard's, coded with the table of a larger vector (section 1.6) */
+  uint32_t cached_lengths; /* 1 if the code lengths came from a length cache (format section 1.7) */
 } lc_info;
 
 /* Library version (major*100 + minor). */
@@ -132,6 +133,26 @@ int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbit
 int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                     uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
                     uint32_t options, lc_cuda_stream_t cs);
+
+/*
+ * lc_compress / lc_compress_update with the code table of an earlier snapshot (Section 3.2, "Huffman Code Table
+ * Caching": when the number of buckets is the same as before, the table is used again, the buckets only being
+ * sorted by their numbers of entries). The cache is the caller's: LC_LENGTH_CACHE_BYTES of DEVICE memory, 16-byte
+ * aligned, all zero before its first use, passed to every call that should share it; the calls that share one
+ * cache must be ordered (same CUDA stream, or events). Format section 1.7 defines its rows and the rule: with u
+ * used symbols, a valid row u - 1 gives the r-th most frequent symbol the row's r-th length, provided the payload
+ * then stays within n * nbits bits; otherwise the Huffman lengths are built as usual and stored in the row.
+ * A stream coded with cached lengths has `cached_lengths` set in its lc_info, is read by lc_recover like any other,
+ * and recovers exactly the state the plain stream recovers; only its size may be larger, since the code is the
+ * optimal one of another snapshot. On this hardware the table pass is about 1 % of the call, so the cache saves
+ * next to nothing here: it is provided because the paper's system has it.
+ * tracked_out   NULL for lc_compress's behaviour, else as for lc_compress_update.
+ * length_cache  NULL or misaligned returns LC_ERR_ARG.
+ */
+#define LC_LENGTH_CACHE_BYTES 262144u
+int lc_compress_cached(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                       uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
+                       void* length_cache, lc_cuda_stream_t cs);
 
 /*
  * Recovery pass (Algorithm 1 step 7 applied k times; u_t = u_0 + sum_i quantized delta_i).

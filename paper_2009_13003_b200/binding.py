@@ -18,7 +18,7 @@ MAX_CHAIN = 8
 
 SYMBOLS = (
     "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_update", "lc_compress_timed",
-    "lc_recover", "lc_compress_opt", "lc_debug_compress_wait", "lc_merge", "lc_compress_async", "lc_shard_stats", "lc_shard_encode",
+    "lc_recover", "lc_compress_opt", "lc_compress_cached", "lc_debug_compress_wait", "lc_merge", "lc_compress_async", "lc_shard_stats", "lc_shard_encode",
     "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
     "lc_debug_bins", "lc_debug_codes", "lc_compress_noalloc",
 )
@@ -30,6 +30,7 @@ class LCInfo(C.Structure):
         ("n", C.c_uint64), ("total_bytes", C.c_uint64), ("payload_bits", C.c_uint64),
         ("payload_offset", C.c_uint64), ("nbits", C.c_uint32), ("nsym", C.c_uint32),
         ("max_len", C.c_uint32), ("nchunks", C.c_uint32), ("valid", C.c_int32), ("fixed_width", C.c_uint32), ("shard", C.c_uint32),
+        ("cached_lengths", C.c_uint32),
     ]
 
 
@@ -65,6 +66,7 @@ def lib():
     L.lc_compress.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp]
     L.lc_compress_update.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
     L.lc_compress_opt.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, C.c_uint32, vp]
+    L.lc_compress_cached.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp, vp]
     L.lc_debug_compress_wait.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, C.c_uint32, C.c_uint32, vp]
     L.lc_compress_timed.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, C.POINTER(C.c_float)]
     L.lc_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
@@ -193,6 +195,35 @@ def compress(base, cur, nbits, stream=None, workspace=None, fixed=False):
     _check(last_status(workspace), "lc_compress (device)")
     info = stream_info(stream)
     return stream[: info.total_bytes]
+
+
+LENGTH_CACHE_BYTES = 262144
+
+
+def alloc_length_cache(device):
+    """An empty length cache for compress_cached (Section 3.2, "Huffman Code Table Caching")."""
+    return torch.zeros(LENGTH_CACHE_BYTES, dtype=torch.uint8, device=device)
+
+
+def compress_cached_async(base, cur, nbits, stream, workspace, length_cache, tracked_out=None):
+    """lc_compress_cached on the current stream; no synchronisation."""
+    _f32_cuda(base, "base"), _f32_cuda(cur, "cur")
+    rc = lib().lc_compress_cached(base.data_ptr(), cur.data_ptr(), base.numel(), nbits, stream.data_ptr(), stream.numel(),
+                                  tracked_out.data_ptr() if tracked_out is not None else None, workspace.data_ptr(),
+                                  workspace.numel(), length_cache.data_ptr(), _cs(base.device))
+    _check(rc, "lc_compress_cached")
+
+
+def compress_cached(base, cur, nbits, length_cache, stream=None, workspace=None, tracked_out=None):
+    """stream <- LC(cur - base), code lengths taken from / stored in ``length_cache`` (changed in place)."""
+    n = base.numel()
+    if stream is None:
+        stream = alloc_stream(n, nbits, base.device)
+    if workspace is None:
+        workspace = alloc_workspace(n, base.device)
+    compress_cached_async(base, cur, nbits, stream, workspace, length_cache, tracked_out)
+    _check(last_status(workspace), "lc_compress_cached (device)")
+    return stream[: stream_info(stream).total_bytes]
 
 
 def compress_update(base, cur, nbits, tracked_out=None, stream=None, workspace=None):

@@ -44,7 +44,7 @@ int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, vo
   cudaError_t e = cudaMemsetAsync(static_cast<uint8_t*>(workspace) + skip, 0, W.plane_off - skip, cs);
   if (e != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, opt.fixed_width, nullptr, cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, opt.fixed_width, nullptr, opt.length_cache, cs)) != cudaSuccess) return LC_ERR_CUDA;
   if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), tracked_out, opt,
                          cs)) != cudaSuccess)
     return LC_ERR_CUDA;
@@ -116,6 +116,19 @@ int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, 
   return compress_impl(base, cur, n, nbits, stream, stream_capacity, tracked_out, workspace, workspace_bytes, opt, cs);
 }
 
+int lc_compress_cached(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
+                       uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
+                       void* length_cache, lc_cuda_stream_t cs) {
+  if (!length_cache || !aligned(length_cache, 16)) return LC_ERR_ARG;
+  if (tracked_out) {
+    const int rc = check_tracked_out(cur, n, tracked_out);
+    if (rc != LC_OK) return rc;
+  }
+  EncodeOptions opt;
+  opt.length_cache = static_cast<uint8_t*>(length_cache);
+  return compress_impl(base, cur, n, nbits, stream, stream_capacity, tracked_out, workspace, workspace_bytes, opt, cs);
+}
+
 int lc_debug_compress_wait(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                            uint64_t stream_capacity, void* workspace, uint64_t workspace_bytes, uint32_t spin_limit,
                            uint32_t first_ticket, lc_cuda_stream_t cs) {
@@ -143,7 +156,7 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
   ok = ok && cudaEventRecord(ev[0], cs) == cudaSuccess;
   ok = ok && launch_stats(base, cur, n, c.ctl, c.plane, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[1], cs) == cudaSuccess;
-  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, false, nullptr, cs) == cudaSuccess;
+  ok = ok && launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, false, nullptr, nullptr, cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[2], cs) == cudaSuccess;
   ok = ok && launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(), cs) == cudaSuccess;
   ok = ok && cudaEventRecord(ev[3], cs) == cudaSuccess;
@@ -197,7 +210,7 @@ int lc_compress_async(const float* base, const float* cur, uint64_t n, int nbits
   if (cudaEventRecord(state_read, cs_state) != cudaSuccess) return LC_ERR_CUDA;
   // beside whatever cs_state does next: table and encode, which work on the bucket statistics and the key plane
   if (cudaStreamWaitEvent(cs_side, state_read, 0) != cudaSuccess) return LC_ERR_CUDA;
-  if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), /*wide_ok=*/false, false, nullptr, cs_side) != cudaSuccess)
+  if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), /*wide_ok=*/false, false, nullptr, nullptr, cs_side) != cudaSuccess)
     return LC_ERR_CUDA;
   if (launch_encode(c.ctl, c.tiles, c.plane, nullptr, nullptr, n, static_cast<uint8_t*>(stream), nullptr,
                     EncodeOptions(), cs_side) != cudaSuccess)
@@ -234,7 +247,7 @@ int lc_shard_encode(const float* base, const float* cur, uint64_t n, int nbits, 
   if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
   const Carved c = carve(workspace, W);
   if (launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, false,
-                   static_cast<const ShardStats*>(whole_stats), cs) != cudaSuccess)
+                   static_cast<const ShardStats*>(whole_stats), nullptr, cs) != cudaSuccess)
     return LC_ERR_CUDA;
   if (launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(),
                     cs) != cudaSuccess)
@@ -273,6 +286,7 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
   info->nbits = h[6];
   info->fixed_width = h[7] & 1u;
   info->shard = (h[7] >> 1) & 1u;
+  info->cached_lengths = (h[7] >> 2) & 1u;
   info->n = le(8, 8);
   info->nsym = (uint32_t)le(16, 4);
   info->max_len = (uint32_t)le(20, 4);
@@ -280,7 +294,7 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
   info->payload_bits = le(40, 8);
   info->total_bytes = le(48, 8);
   info->payload_offset = le(56, 8);
-  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 && h[7] <= 3 &&
+  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 && h[7] <= 4 &&
                  le(24, 4) == kChunkElems && le(28, 2) == kLanes && le(30, 2) == kGroup &&
                  le(36, 4) == kPayloadAlign)
                     ? 1

@@ -133,7 +133,11 @@ struct EncodeOptions {
   uint32_t spin_limit = 1u << 20; // polls of the look-back before it gives up with LC_ERR_TIMEOUT
   uint32_t ticket_bias = 0;       // added to every tile ticket (test aid: with 1, tile 0 is never coded)
   bool fixed_width = false;       // fixed-width codes (format section 1.5) instead of the Huffman code
+  uint8_t* length_cache = nullptr;  // DEVICE, kLengthCacheBytes: code lengths of earlier calls (format section 1.7)
 };
+
+constexpr uint32_t kLengthCacheRow = 512;                            // bytes per row: one row per number of used symbols
+constexpr uint64_t kLengthCacheBytes = 512ull * kLengthCacheRow;
 
 // ---- launchers (each defined next to its kernel) ---------------------------------------------------
 cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
@@ -144,7 +148,7 @@ cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Contro
 // whole: nullptr, or the statistics of the whole vector of which this call codes a shard (format section 1.6):
 //        kept buckets, representatives and code then come from them, the table's counts from ctl's own
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, bool fixed,
-                         const ShardStats* whole, cudaStream_t cs);
+                         const ShardStats* whole, uint8_t* length_cache, cudaStream_t cs);
 // tracked_out: nullptr, or where to write base + quantized delta (may be base itself)
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
                           const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, const EncodeOptions& opt,

@@ -59,7 +59,7 @@ extern "C" int lc_compress_noalloc(const float* base, const float* cur, uint64_t
   // the array keeps what the previous call left: counters, bins and tile descriptors must start at zero
   if (cudaMemsetAsync(w, 0, W.plane_off, cs) != cudaSuccess) return LC_ERR_CUDA;
   if (launch_stats(base, cur, n, ctl, plane, cs) != cudaSuccess) return LC_ERR_CUDA;
-  if (launch_table(ctl, n, nbits, static_cast<uint8_t*>(stream), true, false, nullptr, cs) != cudaSuccess) return LC_ERR_CUDA;
+  if (launch_table(ctl, n, nbits, static_cast<uint8_t*>(stream), true, false, nullptr, nullptr, cs) != cudaSuccess) return LC_ERR_CUDA;
   if (launch_encode(ctl, tiles, plane, base, cur, n, static_cast<uint8_t*>(stream), nullptr, EncodeOptions(), cs) != cudaSuccess)
     return LC_ERR_CUDA;
   int32_t status = 0;

@@ -21,7 +21,7 @@ __device__ __forceinline__ void store_le(uint8_t* p, uint64_t v, int bytes) {
 
 __global__ void __launch_bounds__(kTableThreads)
 table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restrict__ stream, int wide_ok,
-             int fixed, const ShardStats* __restrict__ whole) {
+             int fixed, const ShardStats* __restrict__ whole, uint8_t* __restrict__ cache) {
   __shared__ uint32_t warp_cand[16];
   __shared__ uint16_t sym_of_key[kKeys];
   __shared__ unsigned long long sym_count[kMaxSym];
@@ -36,6 +36,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
   __shared__ uint16_t canon_order[kMaxSym];
   __shared__ uint32_t s_maxlen;
   __shared__ unsigned long long s_kept_total, s_payload_bits;
+  __shared__ unsigned long long s_cached_bits;  // payload size with the lengths of the cache row
 
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
@@ -98,6 +99,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     s_payload_bits = 0;
     s_maxlen = 0;
     s_whole_total = 0;
+    s_cached_bits = 0;
   }
   sym_local[tid] = 0;
   const uint32_t ballot = __ballot_sync(0xffffffffu, cand);
@@ -162,7 +164,29 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
       s_payload_bits = n * width;
     }
   }
-  if (used && !fixed) {
+  // ---- code-table caching (Section 3.2; format section 1.7): a valid row for this number of used symbols gives
+  // the r-th most frequent symbol its r-th length, if the payload then stays within n * nbits bits
+  uint8_t* row = (cache && !fixed && nused >= 2) ? cache + (size_t)kLengthCacheRow * (nused - 1) : nullptr;
+  uint32_t offered = 0;
+  if (row && row[0] != 0 && used) {  // row[0] is read before anything in this kernel writes the row
+    uint32_t r = 0;
+    for (uint32_t j = 0; j < nsym; ++j) {
+      const unsigned long long cj = sym_count[j];
+      if (cj != 0 && (cj > my_count || (cj == my_count && (int)j < tid))) r += 1;
+    }
+    offered = row[r];
+    atomicAdd(&s_cached_bits, my_count * offered);
+  }
+  const bool row_valid = row && row[0] != 0;
+  __syncthreads();
+  const bool hit = row_valid && s_cached_bits <= n * (unsigned long long)nbits;
+  if (hit) {
+    if (used) {
+      sym_len[tid] = offered;
+      atomicMax(&s_maxlen, offered);
+    }
+  }
+  if (used && !fixed && !hit) {
     uint32_t r = 0;
     for (uint32_t j = 0; j < nsym; ++j) {
       const unsigned long long cj = sym_count[j];
@@ -172,7 +196,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     leaf_sym[r] = (uint16_t)tid;
   }
   __syncthreads();
-  if (tid == 0 && nused >= 2 && !fixed) {
+  if (tid == 0 && nused >= 2 && !fixed && !hit) {
     uint32_t front_a = 0, front_b = nused, next = nused;
     for (uint32_t merge = 0; merge + 1 < nused; ++merge) {
       uint32_t pick[2];
@@ -211,7 +235,9 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
       if (lj != 0 && (lj < my_len || (lj == my_len && (int)j < tid))) r += 1;
     }
     canon_order[r] = (uint16_t)tid;
+    if (row && !hit) row[r] = (uint8_t)my_len;  // a miss stores the new lengths, ascending
   }
+  if (row && !hit && tid >= (int)nused) row[tid] = 0;
   __syncthreads();
   if (tid == 0 && nused >= 2 && !fixed) {
     unsigned long long code = 0;
@@ -259,7 +285,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
     store_le(h + 4, 1, 2);
     h[6] = (uint8_t)nbits;
-    h[7] = (uint8_t)((fixed ? 1 : 0) | (whole ? 2 : 0));
+    h[7] = (uint8_t)((fixed ? 1 : 0) | (whole ? 2 : 0) | (hit ? 4 : 0));
     store_le(h + 8, n, 8);
     store_le(h + 16, nsym, 4);
     store_le(h + 20, s_maxlen, 4);
@@ -283,8 +309,8 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
 }  // namespace
 
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, bool fixed,
-                         const ShardStats* whole, cudaStream_t cs) {
-  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0, fixed ? 1 : 0, whole);
+                         const ShardStats* whole, uint8_t* cache, cudaStream_t cs) {
+  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0, fixed ? 1 : 0, whole, cache);
   return cudaGetLastError();
 }
 
