@@ -400,6 +400,11 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
   }
   const uint64_t e0 = c * kChunkElems + 4 * lane;
   float4 b = ldg_stream_v4(base + e0);
+  // With one stream a step is short, and one row of base in registers ahead of its use leaves too few bytes in flight
+  // for the L2's latency (0.80 of the copy rate); a second row brings that to 0.92. With two or more streams the
+  // second row makes the kernel slower (measured for 2, 3 and 4 streams), so they keep one.
+  float4 b2 = b;
+  if (KS == 1) b2 = ldg_stream_v4(base + e0 + 128);
   // Rows of base are asked into the L2 kPrefetchRows steps before they are loaded: a warp has one row in
   // registers ahead of its use, which alone leaves far too few bytes in flight per SM for the DRAM latency.
   // Behind this chunk's last row the requests go on with the first rows of the chunk this warp decodes next
@@ -409,8 +414,14 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
   for (uint32_t j = 0; j < kSteps; ++j) {
     const uint64_t i = e0 + 128ull * j;
     float x[4] = {b.x, b.y, b.z, b.w};
-    // next step's 16 bytes of base, requested a whole step ahead (the last step re-reads its own)
-    b = ldg_stream_v4(base + i + (j + 1 < kSteps ? 128 : 0));
+    // the 16 bytes of base of a later step, requested one step ahead (one stream: two steps); the last steps
+    // re-read their own
+    if (KS == 1) {
+      b = b2;
+      b2 = ldg_stream_v4(base + i + (j + 2 < kSteps ? 256 : 0));
+    } else {
+      b = ldg_stream_v4(base + i + (j + 1 < kSteps ? 128 : 0));
+    }
     asm volatile("prefetch.global.L2 [%0];" ::"l"(pf));
     pf = (j == kSteps - kPrefetchRows - 1) ? next_rows : pf + 128;
     int cnt0[KS];
