@@ -489,6 +489,39 @@ def run_ours(args, rank, world, local_rank):
               "bytes_vs_plain": int(info_c.total_bytes) / stream_bytes[-1]}
     del cache
 
+    # ---- per-layer granularity on the workload that has layers (ResNet-18-sized: 62 segments): one stream per
+    # segment against one stream for the flat vector; outside the timed region
+    per_layer = None
+    if cfg.name == "resnet18" and n == cfg.n:
+        begin = [0]
+        for size in synth.resnet18_segments():
+            begin.append(begin[-1] + size)
+        seg_offsets, seg_total = lc.segments_layout(begin, nbits)
+        seg_streams = torch.empty(seg_total, dtype=torch.uint8, device=dev)
+        seg_out = torch.empty_like(u0)
+        tc, tr = [], []
+        for it in range(6):
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record()
+            lc.compress_segments_async(tracked, u, begin, nbits, seg_streams, ws)
+            e[1].record()
+            lc.recover_segments_async(tracked, [seg_streams], begin, nbits, seg_out, ws)
+            e[2].record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                tc.append(e[0].elapsed_time(e[1]))
+                tr.append(e[1].elapsed_time(e[2]))
+        assert lc.last_status(ws) == 0
+        seg_bytes = sum(int(lc.stream_info(seg_streams[o:]).total_bytes) for o in seg_offsets[:-1])
+        flat_out = lc.recover(tracked, [streams[-1]])
+        flat_err = float((flat_out - u).abs().double().sum())
+        del flat_out
+        seg_err = float((seg_out - u).abs().double().sum())
+        per_layer = {"segments": len(begin) - 1, "compress_ms": statistics.median(tc), "recover_ms": statistics.median(tr),
+                     "ratio": 4.0 * n / seg_bytes, "flat_ratio": 4.0 * n / stream_bytes[-1],
+                     "abs_error_vs_flat": seg_err / flat_err if flat_err else None}
+        del seg_streams, seg_out
+
     # ---- end to end through the host-buffer entry points (pinned host memory, copies inside)
     e2e = None
     if chain <= lc.MAX_CHAIN:
@@ -566,6 +599,7 @@ def run_ours(args, rank, world, local_rank):
                             "alg_gbs": (12.0 * n + stream_bytes[-1]) / (cu_ms * 1e-3) / 1e9,
                             "frac_of_peak": (12.0 * n + stream_bytes[-1]) / (cu_ms * 1e-3) / 1e9 / peak},
         "table_caching": cached,
+        "per_layer": per_layer,
         # algorithmic bytes of a merge: read base and the chain's streams, write the merged stream
         "merge": None if merge_ms is None else {
             "ms": merge_ms, "streams_in": chain, "merged_ratio": 4.0 * n / merged_bytes,

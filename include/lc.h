@@ -135,6 +135,35 @@ int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, 
                     uint32_t options, lc_cuda_stream_t cs);
 
 /*
+ * Per-layer granularity. The paper compresses "the model state"; whether layer by layer or as one vector it does not
+ * say. These calls cut the vector into nseg contiguous segments (the layers of a model) and code every segment as a
+ * complete stream of its own, with its own buckets, representatives and code (Sections 3.1.1 and 3.1.2 applied per
+ * segment): layers whose updates differ in scale then each keep their own top 2^nbits - 1 buckets. Each segment's
+ * stream is byte for byte what lc_compress writes for that slice of base and cur.
+ * seg_begin     HOST, nseg + 1 element offsets, seg_begin[0] = 0, non-decreasing, every one a multiple of 4 (the
+ *               segments then start on 16-byte boundaries), each segment shorter than 2^32 elements;
+ *               1 <= nseg <= LC_MAX_SEGMENTS. The vector has seg_begin[nseg] elements.
+ * lc_segments_layout: where the streams go. Segment i's stream starts at byte stream_offset[i] of the streams buffer
+ *               (its slot ends at stream_offset[i + 1]: lc_stream_bound of the segment, rounded up to 256);
+ *               stream_offset (HOST, nseg + 1 entries) may be NULL. Returns the buffer size needed, 0 on bad arguments.
+ * streams       DEVICE, 256-byte aligned, streams_capacity >= lc_segments_layout(...). For lc_recover_segments: HOST
+ *               array of k such buffers, applied in array order (1 <= k <= LC_MAX_CHAIN).
+ * tracked_out   NULL, or as for lc_compress_update (the whole vector; may be base).
+ * workspace     as for lc_compress, of lc_workspace_bytes(longest segment) bytes; one status word for the call: the
+ *               first failure of any segment stays in it (lc_last_status), and the segments after a failed one are
+ *               left without a valid stream (compress) or with unspecified output (recover).
+ * The segments run one after the other on `cs`, a handful of launches each: this is for models of tens to hundreds
+ * of layers, not for millions of tiny tensors.
+ */
+#define LC_MAX_SEGMENTS 65536
+uint64_t lc_segments_layout(const uint64_t* seg_begin, int nseg, int nbits, uint64_t* stream_offset);
+int lc_compress_segments(const float* base, const float* cur, const uint64_t* seg_begin, int nseg, int nbits,
+                         void* streams, uint64_t streams_capacity, float* tracked_out, void* workspace,
+                         uint64_t workspace_bytes, lc_cuda_stream_t cs);
+int lc_recover_segments(const float* base, const void* const* streams, int k, const uint64_t* seg_begin, int nseg,
+                        int nbits, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs);
+
+/*
  * lc_compress / lc_compress_update with the code table of an earlier snapshot (Section 3.2, "Huffman Code Table
  * Caching": when the number of buckets is the same as before, the table is used again, the buckets only being
  * sorted by their numbers of entries). The cache is the caller's: LC_LENGTH_CACHE_BYTES of DEVICE memory, 16-byte

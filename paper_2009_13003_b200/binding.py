@@ -18,7 +18,8 @@ MAX_CHAIN = 8
 
 SYMBOLS = (
     "lc_version", "lc_strerror", "lc_stream_bound", "lc_workspace_bytes", "lc_compress", "lc_compress_update", "lc_compress_timed",
-    "lc_recover", "lc_compress_opt", "lc_compress_cached", "lc_debug_compress_wait", "lc_merge", "lc_compress_async", "lc_shard_stats", "lc_shard_encode",
+    "lc_recover", "lc_compress_opt", "lc_compress_cached",
+    "lc_segments_layout", "lc_compress_segments", "lc_recover_segments", "lc_debug_compress_wait", "lc_merge", "lc_compress_async", "lc_shard_stats", "lc_shard_encode",
     "lc_stream_info", "lc_last_status", "lc_host_arena_bytes", "lc_compress_host", "lc_recover_host",
     "lc_debug_bins", "lc_debug_codes", "lc_compress_noalloc",
 )
@@ -67,6 +68,10 @@ def lib():
     L.lc_compress_update.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
     L.lc_compress_opt.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, C.c_uint32, vp]
     L.lc_compress_cached.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp, vp]
+    L.lc_segments_layout.argtypes = [C.POINTER(u64), i32, i32, C.POINTER(u64)]
+    L.lc_segments_layout.restype = u64
+    L.lc_compress_segments.argtypes = [vp, vp, C.POINTER(u64), i32, i32, vp, u64, vp, vp, u64, vp]
+    L.lc_recover_segments.argtypes = [vp, C.POINTER(vp), i32, C.POINTER(u64), i32, i32, vp, vp, u64, vp]
     L.lc_debug_compress_wait.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, C.c_uint32, C.c_uint32, vp]
     L.lc_compress_timed.argtypes = [vp, vp, u64, i32, vp, u64, vp, u64, vp, C.POINTER(C.c_float)]
     L.lc_recover.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, vp, vp, u64, vp]
@@ -224,6 +229,62 @@ def compress_cached(base, cur, nbits, length_cache, stream=None, workspace=None,
     compress_cached_async(base, cur, nbits, stream, workspace, length_cache, tracked_out)
     _check(last_status(workspace), "lc_compress_cached (device)")
     return stream[: stream_info(stream).total_bytes]
+
+
+def segments_layout(seg_begin, nbits):
+    """(stream offsets, total bytes) of the streams buffer for the segments that start at ``seg_begin`` (nseg + 1
+    element offsets)."""
+    nseg = len(seg_begin) - 1
+    sb = (C.c_uint64 * (nseg + 1))(*seg_begin)
+    off = (C.c_uint64 * (nseg + 1))()
+    total = int(lib().lc_segments_layout(sb, nseg, nbits, off))
+    if total == 0 and nseg > 0:
+        raise LCError(ERR_ARG, "lc_segments_layout")
+    return [int(x) for x in off], total
+
+
+def compress_segments_async(base, cur, seg_begin, nbits, streams, workspace, tracked_out=None):
+    """lc_compress_segments on the current stream; no synchronisation."""
+    _f32_cuda(base, "base"), _f32_cuda(cur, "cur")
+    nseg = len(seg_begin) - 1
+    sb = (C.c_uint64 * (nseg + 1))(*seg_begin)
+    rc = lib().lc_compress_segments(base.data_ptr(), cur.data_ptr(), sb, nseg, nbits, streams.data_ptr(), streams.numel(),
+                                    tracked_out.data_ptr() if tracked_out is not None else None, workspace.data_ptr(),
+                                    workspace.numel(), _cs(base.device))
+    _check(rc, "lc_compress_segments")
+
+
+def compress_segments(base, cur, seg_begin, nbits, streams=None, workspace=None, tracked_out=None):
+    """One stream per segment. Returns (streams buffer, offsets): segment i's stream starts at offsets[i]."""
+    offsets, total = segments_layout(seg_begin, nbits)
+    if streams is None:
+        streams = torch.empty(total, dtype=torch.uint8, device=base.device)
+    if workspace is None:
+        longest = max([b - a for a, b in zip(seg_begin[:-1], seg_begin[1:])] + [0])
+        workspace = alloc_workspace(longest, base.device)
+    compress_segments_async(base, cur, seg_begin, nbits, streams, workspace, tracked_out)
+    _check(last_status(workspace), "lc_compress_segments (device)")
+    return streams, offsets
+
+
+def recover_segments_async(base, streams_list, seg_begin, nbits, out, workspace):
+    """lc_recover_segments on the current stream; ``streams_list``: the buffers of a chain, in order."""
+    nseg, k = len(seg_begin) - 1, len(streams_list)
+    sb = (C.c_uint64 * (nseg + 1))(*seg_begin)
+    ptrs = (C.c_void_p * k)(*[s.data_ptr() for s in streams_list])
+    rc = lib().lc_recover_segments(base.data_ptr(), ptrs, k, sb, nseg, nbits, out.data_ptr(), workspace.data_ptr(),
+                                   workspace.numel(), _cs(base.device))
+    _check(rc, "lc_recover_segments")
+
+
+def recover_segments(base, streams_list, seg_begin, nbits, out=None, workspace=None):
+    if out is None:
+        out = torch.empty_like(base)
+    if workspace is None:
+        workspace = alloc_workspace(0, base.device)
+    recover_segments_async(base, streams_list, seg_begin, nbits, out, workspace)
+    _check(last_status(workspace), "lc_recover_segments (device)")
+    return out
 
 
 def compress_update(base, cur, nbits, tracked_out=None, stream=None, workspace=None):

@@ -166,8 +166,10 @@ int lc_compress_timed(const float* base, const float* cur, uint64_t n, int nbits
   return ok ? LC_OK : LC_ERR_CUDA;
 }
 
-int lc_recover(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k,
-               uint64_t n, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+// lc_recover; reset_status: false when an earlier part of the same call may already have set the status word
+static int recover_impl(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k,
+                        uint64_t n, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs,
+                        bool reset_status) {
   if (k < 1 || k > LC_MAX_CHAIN || n >= (1ull << 32)) return LC_ERR_ARG;
   if (!streams || !stream_bytes || !workspace || (n > 0 && (!base || !out))) return LC_ERR_ARG;
   if (!aligned(base, 16) || !aligned(out, 16) || !aligned(workspace, 256)) return LC_ERR_ARG;
@@ -176,8 +178,7 @@ int lc_recover(const float* base, const void* const* streams, const uint64_t* st
   if (workspace_bytes < workspace_layout(0).total) return LC_ERR_CAPACITY;
   Control* ctl = static_cast<Control*>(workspace);
   void* images = static_cast<uint8_t*>(workspace) + workspace_layout(0).decode_off;
-  cudaError_t e = cudaMemsetAsync(&ctl->status, 0, sizeof(int32_t), cs);
-  if (e != cudaSuccess) return LC_ERR_CUDA;
+  if (reset_status && cudaMemsetAsync(&ctl->status, 0, sizeof(int32_t), cs) != cudaSuccess) return LC_ERR_CUDA;
   // up to four streams per launch; later launches continue in place from `out`.
   const float* src = base;
   for (int first = 0; first < k; first += 4) {
@@ -188,8 +189,83 @@ int lc_recover(const float* base, const void* const* streams, const uint64_t* st
       ds.ptr[j] = static_cast<const uint8_t*>(streams[first + j]);
       ds.bytes[j] = stream_bytes[first + j];
     }
-    if ((e = launch_decode(src, ds, kk, n, out, &ctl->status, images, cs)) != cudaSuccess) return LC_ERR_CUDA;
+    if (launch_decode(src, ds, kk, n, out, &ctl->status, images, cs) != cudaSuccess) return LC_ERR_CUDA;
     src = out;
+  }
+  return LC_OK;
+}
+
+int lc_recover(const float* base, const void* const* streams, const uint64_t* stream_bytes, int k,
+               uint64_t n, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+  return recover_impl(base, streams, stream_bytes, k, n, out, workspace, workspace_bytes, cs, true);
+}
+
+// ---- per-layer granularity: one stream per segment of the vector --------------------------------------------
+
+static bool segments_ok(const uint64_t* seg_begin, int nseg) {
+  if (!seg_begin || nseg < 1 || nseg > LC_MAX_SEGMENTS || seg_begin[0] != 0) return false;
+  for (int i = 0; i < nseg; ++i)
+    if (seg_begin[i + 1] < seg_begin[i] || (seg_begin[i + 1] & 3u) != 0 || seg_begin[i + 1] - seg_begin[i] >= (1ull << 32))
+      return false;
+  return true;
+}
+
+uint64_t lc_segments_layout(const uint64_t* seg_begin, int nseg, int nbits, uint64_t* stream_offset) {
+  if (!segments_ok(seg_begin, nseg) || nbits < 1 || nbits > kMaxNbits) return 0;
+  uint64_t off = 0;
+  for (int i = 0; i < nseg; ++i) {
+    if (stream_offset) stream_offset[i] = off;
+    off += align_up(lc_stream_bound(seg_begin[i + 1] - seg_begin[i], nbits), 256);
+  }
+  if (stream_offset) stream_offset[nseg] = off;
+  return off;
+}
+
+int lc_compress_segments(const float* base, const float* cur, const uint64_t* seg_begin, int nseg, int nbits,
+                         void* streams, uint64_t streams_capacity, float* tracked_out, void* workspace,
+                         uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+  if (!segments_ok(seg_begin, nseg) || nbits < 1 || nbits > kMaxNbits || !streams || !aligned(streams, 256))
+    return LC_ERR_ARG;
+  if (streams_capacity < lc_segments_layout(seg_begin, nseg, nbits, nullptr)) return LC_ERR_CAPACITY;
+  uint64_t off = 0;
+  for (int i = 0; i < nseg; ++i) {
+    const uint64_t lo = seg_begin[i], ni = seg_begin[i + 1] - lo;
+    const uint64_t cap = align_up(lc_stream_bound(ni, nbits), 256);
+    float* t = tracked_out ? tracked_out + lo : nullptr;
+    if (t) {
+      const int rc = check_tracked_out(cur + lo, ni, t);
+      if (rc != LC_OK) return rc;
+    }
+    // the status word is cleared before the first segment only: a segment the device rejects makes the table and
+    // encode passes of all later ones leave their streams invalid, and the word keeps the first failure
+    const int rc = compress_impl(base + lo, cur + lo, ni, nbits, static_cast<uint8_t*>(streams) + off, cap, t, workspace,
+                                 workspace_bytes, EncodeOptions(), cs, /*keep_status=*/i > 0);
+    if (rc != LC_OK) return rc;
+    off += cap;
+  }
+  return LC_OK;
+}
+
+int lc_recover_segments(const float* base, const void* const* streams, int k, const uint64_t* seg_begin, int nseg,
+                        int nbits, float* out, void* workspace, uint64_t workspace_bytes, lc_cuda_stream_t cs) {
+  if (!segments_ok(seg_begin, nseg) || nbits < 1 || nbits > kMaxNbits || k < 1 || k > LC_MAX_CHAIN || !streams)
+    return LC_ERR_ARG;
+  for (int j = 0; j < k; ++j)
+    if (!streams[j] || !aligned(streams[j], 256)) return LC_ERR_ARG;
+  uint64_t off = 0;
+  for (int i = 0; i < nseg; ++i) {
+    const uint64_t lo = seg_begin[i], ni = seg_begin[i + 1] - lo;
+    const uint64_t cap = align_up(lc_stream_bound(ni, nbits), 256);
+    const void* seg_streams[LC_MAX_CHAIN];
+    uint64_t seg_bytes[LC_MAX_CHAIN];
+    for (int j = 0; j < k; ++j) {
+      seg_streams[j] = static_cast<const uint8_t*>(streams[j]) + off;
+      seg_bytes[j] = cap;
+    }
+    const int rc = recover_impl(base + lo, seg_streams, seg_bytes, k, ni, out + lo, workspace, workspace_bytes, cs,
+                                /*reset_status=*/i == 0);
+    if (rc != LC_OK) return rc;
+    off += cap;
   }
   return LC_OK;
 }

@@ -51,7 +51,10 @@ static_assert(((1 << kL1Bits) << (kSubBitsMin + 3)) <= 8192, "at the smallest de
 // which is how the hot loop notices: a step subtracts at most four of them per stream, and 1..4 times 2^29 (less a
 // few real lengths) leaves the sign bit of the 32-bit count set in every case.
 constexpr uint32_t kLongCode = 0x20000000u;
-constexpr int kPrefetchRows = 8;  // distance, in steps of 512 bytes per warp, of the L2 prefetch of base
+// distance, in steps of 512 bytes per warp, of the L2 prefetch of base (measured: 4, 6, 8, 12 and 16 rows; chains of
+// two and more do not care between 4 and 12, a single stream is fastest at 6)
+template <int KS>
+constexpr int kPrefetchRows = KS == 1 ? 6 : 8;
 
 // The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory.
 constexpr uint32_t kTableBytes = 8192;
@@ -409,7 +412,7 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
   // registers ahead of its use, which alone leaves far too few bytes in flight per SM for the DRAM latency.
   // Behind this chunk's last row the requests go on with the first rows of the chunk this warp decodes next
   // (`next_rows`: this lane's part of that chunk's first row, or of this chunk's first row if there is none).
-  const float* pf = base + e0 + 128 * kPrefetchRows;
+  const float* pf = base + e0 + 128 * kPrefetchRows<KS>;
 #pragma unroll 1
   for (uint32_t j = 0; j < kSteps; ++j) {
     const uint64_t i = e0 + 128ull * j;
@@ -423,7 +426,7 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
       b = ldg_stream_v4(base + i + (j + 1 < kSteps ? 128 : 0));
     }
     asm volatile("prefetch.global.L2 [%0];" ::"l"(pf));
-    pf = (j == kSteps - kPrefetchRows - 1) ? next_rows : pf + 128;
+    pf = (j == kSteps - kPrefetchRows<KS> - 1) ? next_rows : pf + 128;
     int cnt0[KS];
     uint32_t next0[KS];
     uint32_t flags = 0;
