@@ -19,7 +19,9 @@
 // base (the merged stream of one stream is that stream) and to Algorithm 1 step 7 applied to the
 // recovered state. The length cache of Section 3.2 (lco_cached_lengths, lco_compress_cached) is pinned by hand-worked
 // rows and assignments, by byte equality with the plain stream on an empty cache, and by a cached stream
-// recovering the plain stream's state with more payload bits than the plain stream's optimal code.
+// recovering the plain stream's state with more payload bits than the plain stream's optimal code. The mean
+// variant (lco_bucket_mean, lco_compress_mean) is pinned by hand-worked buckets (ties, thirds of an ulp, both ends
+// of the exponent range) and by exact rational arithmetic on random buckets and on the buckets of a stream.
 // Parity unpinned: the whole-pipeline result on the paper's own training deltas (its figures carry
 // the only values and they are not available); only the loose size ranges of Section 4.3 apply.
 
@@ -72,6 +74,7 @@ struct Bucket {
   uint64_t count = 0;
   float vmin = 0.0f;  // smallest value seen in the bucket
   float vmax = 0.0f;  // largest value seen in the bucket
+  unsigned __int128 sig_sum = 0;  // sum of the 24-bit integer significands of the bucket's values (mean variant)
 };
 
 // Algorithm 1 step 4 (delta against the tracked state) followed by the bucketing of Section 3.1.1.
@@ -88,7 +91,20 @@ void delta_buckets(const float* base, const float* cur, uint64_t n, Bucket* buck
       if (d > b.vmax) b.vmax = d;
     }
     b.count += 1;
+    b.sig_sum += (float_bits(d) & 0x7FFFFFu) | 0x800000u;
   }
+}
+
+// Variant (format section 1.8): the bucket is represented by the MEAN of its values instead of the average of its
+// maximum and minimum. Every value of a bucket is sign * 2^(E-150) * (its 24-bit integer significand), so the exact
+// mean is that scale times the mean of the integers; rounding the latter to the nearest integer, ties to even,
+// rounds the exact mean to fp32 (the mean lies in the bucket's binade, where fp32 values are those integers).
+float bucket_mean(int key, unsigned __int128 sig_sum, uint64_t count) {
+  const unsigned __int128 q = sig_sum / count, r = sig_sum % count;
+  uint64_t sig = static_cast<uint64_t>(q);
+  if (2 * r > count || (2 * r == count && (sig & 1u))) sig += 1;
+  const double magnitude = std::ldexp(static_cast<double>(sig), (key & 255) - 150);
+  return static_cast<float>((key >> 8) ? -magnitude : magnitude);
 }
 
 struct Selection {
@@ -199,6 +215,7 @@ struct Table {
   int fixed = 0;   // 1: fixed-width codes (format section 1.5) instead of the Huffman code
   int shared = 0;  // 1: the table was built from a larger vector than the stream codes (format section 1.6)
   int cached = 0;  // 1: the code lengths were taken from a length cache (format section 1.7)
+  int mean = 0;    // 1: representatives are bucket means (format section 1.8)
   int key[512] = {};
   int len[512] = {};
   float rep[512] = {};
@@ -247,7 +264,7 @@ int cached_lengths(const uint64_t* count, int nsym, int nbits, uint64_t n, uint8
 }
 
 int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selection* sel_out, int fixed = 0,
-                uint8_t* cache = nullptr) {
+                uint8_t* cache = nullptr, int mean = 0) {
   for (int s = 0; s <= 1; ++s)
     if (buckets[256 * s + 255].count > 0) return LCO_ERR_NONFINITE;
   const Selection sel = priority_promotion(buckets, nbits);
@@ -258,7 +275,7 @@ int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selectio
   for (int j = 1; j < sel.nsym; ++j) {
     const Bucket& b = buckets[sel.key_of_symbol[j]];
     t->key[j] = sel.key_of_symbol[j];
-    t->rep[j] = midrange(b.vmin, b.vmax);
+    t->rep[j] = mean ? bucket_mean(sel.key_of_symbol[j], b.sig_sum, b.count) : midrange(b.vmin, b.vmax);
     t->count[j] = b.count;
     kept_total += b.count;
   }
@@ -266,6 +283,7 @@ int build_table(const Bucket* buckets, uint64_t n, int nbits, Table* t, Selectio
   t->rep[0] = 0.0f;
   t->count[0] = n - kept_total;
   t->fixed = fixed;
+  t->mean = mean;
   if (fixed) {
     // Section 3.1.1's size model: every bucket index takes ceil(log2 k) bits; the code of a symbol is its id.
     int width = 0;
@@ -378,10 +396,10 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   if (!(s[0] == 'L' && s[1] == 'C' && s[2] == 'C' && s[3] == '1')) return LCO_ERR_FORMAT;
   if (get_le(s + 4, 2) != 1) return LCO_ERR_FORMAT;
   const int nbits = static_cast<int>(s[6]);
-  if (nbits < 1 || nbits > 9 || s[7] > 7) return LCO_ERR_FORMAT;
+  if (nbits < 1 || nbits > 9 || s[7] > 15) return LCO_ERR_FORMAT;
   const int fixed = static_cast<int>(s[7] & 1), shared = static_cast<int>((s[7] >> 1) & 1);
-  const int cached = static_cast<int>((s[7] >> 2) & 1);
-  if (cached && (fixed || shared)) return LCO_ERR_FORMAT;
+  const int cached = static_cast<int>((s[7] >> 2) & 1), mean = static_cast<int>((s[7] >> 3) & 1);
+  if ((cached || mean) && (s[7] & (s[7] - 1)) != 0) return LCO_ERR_FORMAT;  // bits 2 and 3 each go alone
   const uint64_t n = get_le(s + 8, 8);
   const uint64_t nsym = get_le(s + 16, 4);
   const uint64_t max_len = get_le(s + 20, 4);
@@ -424,6 +442,7 @@ int parse_stream(const uint8_t* s, uint64_t bytes, Parsed* out) {
   p.table.fixed = fixed;
   p.table.shared = shared;
   p.table.cached = cached;
+  p.table.mean = mean;
   if (fixed) {
     int width = 0;
     while ((1ull << width) < nsym) width += 1;
@@ -560,7 +579,7 @@ void write_header_and_table(uint8_t* stream, const Table& t, uint64_t n, int nbi
   h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
   put_le(h + 4, 1, 2);
   h[6] = static_cast<uint8_t>(nbits);
-  h[7] = static_cast<uint8_t>(t.fixed | (t.shared << 1) | (t.cached << 2));
+  h[7] = static_cast<uint8_t>(t.fixed | (t.shared << 1) | (t.cached << 2) | (t.mean << 3));
   put_le(h + 8, n, 8);
   put_le(h + 16, static_cast<uint64_t>(t.nsym), 4);
   put_le(h + 20, static_cast<uint64_t>(t.max_len), 4);
@@ -673,14 +692,15 @@ uint64_t lco_stream_bound(uint64_t n, int nbits) { return stream_bound(n, nbits)
 // Section 3.1.1 and the "E" / "E+P" stages of Section 4.3's size breakdown).
 // `cache`: null, or the length cache of Section 3.2's "Huffman Code Table Caching" (read and updated).
 static int compress_body(const float* base, const float* cur, uint64_t n, int nbits, int fixed, uint8_t* cache,
-                         uint8_t* stream, uint64_t capacity, uint64_t* out_bytes) {
+                         uint8_t* stream, uint64_t capacity, uint64_t* out_bytes, int mean = 0) {
   if (nbits < 1 || nbits > 9 || fixed < 0 || fixed > 1 || n >= (1ull << 32) || (cache && fixed)) return LCO_ERR_ARG;
+  if (mean && (fixed || cache)) return LCO_ERR_ARG;
   if (capacity < stream_bound(n, nbits)) return LCO_ERR_CAPACITY;
   std::vector<Bucket> buckets(512);
   delta_buckets(base, cur, n, buckets.data());
   Table t;
   Selection sel;
-  const int rc = build_table(buckets.data(), n, nbits, &t, &sel, fixed, cache);
+  const int rc = build_table(buckets.data(), n, nbits, &t, &sel, fixed, cache, mean);
   if (rc != LCO_OK) return rc;
 
   const Layout L = layout_for(n, t.nsym);
@@ -715,6 +735,24 @@ int lco_compress_cached(const float* base, const float* cur, uint64_t n, int nbi
                         uint64_t capacity, uint64_t* out_bytes) {
   if (!cache) return LCO_ERR_ARG;
   return compress_body(base, cur, n, nbits, 0, cache, stream, capacity, out_bytes);
+}
+
+// Compress pass with bucket means as representatives (format section 1.8) instead of Section 3.1.1's midrange.
+int lco_compress_mean(const float* base, const float* cur, uint64_t n, int nbits, uint8_t* stream, uint64_t capacity,
+                      uint64_t* out_bytes) {
+  return compress_body(base, cur, n, nbits, 0, nullptr, stream, capacity, out_bytes, 1);
+}
+
+// The mean of `count` values that share sign and exponent (one bucket), as the mean variant represents them.
+// Returns NaN if they do not form one bucket of normal numbers.
+float lco_bucket_mean(const float* values, uint64_t count) {
+  if (count == 0) return NAN;
+  std::vector<float> zero(count, 0.0f);
+  std::vector<Bucket> buckets(512);
+  delta_buckets(zero.data(), values, count, buckets.data());
+  const int key = bucket_key(values[0] - 0.0f);
+  if (buckets[key].count != count || (key & 255) == 0 || (key & 255) == 255) return NAN;
+  return bucket_mean(key, buckets[key].sig_sum, count);
 }
 
 // The caching step alone: code lengths of `nsym` symbols with the given counts (n = their sum). Returns 1 on a hit.
@@ -843,6 +881,7 @@ int lco_compress_mode_mt(const float* base, const float* cur, uint64_t n, int nb
         m = b;
       } else {
         m.count += b.count;
+        m.sig_sum += b.sig_sum;
         if (b.vmin < m.vmin) m.vmin = b.vmin;
         if (b.vmax > m.vmax) m.vmax = b.vmax;
       }

@@ -40,6 +40,9 @@ def lib():
         L.lco_compress_mode_mt.argtypes = [vp, vp, u64, i32, i32, vp, u64, C.POINTER(u64), i32]
         L.lco_compress_cached.argtypes = [vp, vp, u64, i32, vp, vp, u64, C.POINTER(u64)]
         L.lco_cached_lengths.argtypes = [vp, i32, i32, u64, vp, vp]
+        L.lco_compress_mean.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64)]
+        L.lco_bucket_mean.argtypes = [vp, u64]
+        L.lco_bucket_mean.restype = C.c_float
         L.lco_compress_shard.argtypes = [vp, vp, u64, u64, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_mt.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), i32]
@@ -168,6 +171,25 @@ def cached_lengths(count, nbits, cache):
     hit = lib().lco_cached_lengths(count.ctypes.data, count.size, nbits, int(count.sum()), cache.ctypes.data,
                                    ln.ctypes.data)
     return bool(hit), ln
+
+
+def compress_mean(base, cur, nbits):
+    """Compress pass with bucket means as representatives (format section 1.8)."""
+    base, pb = _f32(base)
+    cur, pc = _f32(cur)
+    cap = stream_bound(base.size, nbits)
+    buf = np.zeros(cap, np.uint8)
+    out = C.c_uint64(0)
+    rc = lib().lco_compress_mean(pb, pc, base.size, nbits, buf.ctypes.data, cap, C.byref(out))
+    if rc < 0:
+        raise OracleError(rc)
+    return buf[: out.value].copy()
+
+
+def bucket_mean(values):
+    """Representative of the mean variant for values that share sign and exponent."""
+    v = np.ascontiguousarray(values, dtype=np.float32)
+    return np.float32(lib().lco_bucket_mean(v.ctypes.data, v.size))
 
 
 def compress_shard(base, cur, lo, hi, nbits):

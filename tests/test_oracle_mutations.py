@@ -67,6 +67,12 @@ MUTATIONS = [
     ("cache: row stored unsorted", "std::sort(sorted.begin(), sorted.end());", ""),
     ("cache: a hit is coded with the Huffman lengths", "if (cache) t->cached = cached_lengths(t->count, t->nsym, nbits, n, cache, t->len);\n    else huffman_lengths(t->count, t->nsym, t->len);",
      "if (cache) { std::vector<int> tmp(512); t->cached = cached_lengths(t->count, t->nsym, nbits, n, cache, tmp.data()); }\n    huffman_lengths(t->count, t->nsym, t->len);"),
+    ("mean: always rounds down", "if (2 * r > count || (2 * r == count && (sig & 1u))) sig += 1;", ""),
+    ("mean: ties away from zero", "(2 * r == count && (sig & 1u))", "(2 * r == count)"),
+    ("mean: implicit leading bit dropped", "b.sig_sum += (float_bits(d) & 0x7FFFFFu) | 0x800000u;", "b.sig_sum += (float_bits(d) & 0x7FFFFFu);"),
+    ("mean: sign dropped", "return static_cast<float>((key >> 8) ? -magnitude : magnitude);", "return static_cast<float>(magnitude);"),
+    ("mean mode still takes the midrange", "t->rep[j] = mean ? bucket_mean(sel.key_of_symbol[j], b.sig_sum, b.count) : midrange(b.vmin, b.vmax);",
+     "t->rep[j] = midrange(b.vmin, b.vmax);"),
     ("size model uses floor log", "while ((1ull << width) < k) width += 1;", "while ((2ull << width) <= k) width += 1;"),
 ]
 
@@ -100,6 +106,9 @@ class _Oracle:
         L.lco_compress_cached.argtypes = [vp, vp, u64, i32, vp, vp, u64, C.POINTER(u64)]
         L.lco_cached_lengths.argtypes = [vp, i32, i32, u64, vp, vp]
         L.lco_apply_quantized.argtypes = [vp, vp, u64, i32, vp]
+        L.lco_compress_mean.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64)]
+        L.lco_bucket_mean.argtypes = [vp, u64]
+        L.lco_bucket_mean.restype = C.c_float
         L.lco_compress_chunks.argtypes = [vp, vp, u64, i32, vp, u64, vp, vp, u64, vp]
         L.lco_merge.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), i32, u64, i32, vp, u64, C.POINTER(u64)]
         L.lco_compress_mt.argtypes = [vp, vp, u64, i32, vp, u64, C.POINTER(u64), i32]
@@ -126,6 +135,18 @@ class _Oracle:
         out = C.c_uint64(0)
         assert self.L.lco_compress_cached(base.ctypes.data, cur.ctypes.data, base.size, nbits, cache.ctypes.data,
                                           buf.ctypes.data, cap, C.byref(out)) == 0
+        return buf[: out.value].copy()
+
+    def bucket_mean(self, values):
+        v = np.ascontiguousarray(values, dtype=np.float32)
+        return np.float32(self.L.lco_bucket_mean(v.ctypes.data, v.size))
+
+    def compress_mean(self, base, cur, nbits):
+        cap = int(self.L.lco_stream_bound(base.size, nbits))
+        buf = np.zeros(cap + 64, np.uint8)
+        out = C.c_uint64(0)
+        assert self.L.lco_compress_mean(base.ctypes.data, cur.ctypes.data, base.size, nbits, buf.ctypes.data, cap,
+                                        C.byref(out)) == 0
         return buf[: out.value].copy()
 
     def compress_shard(self, base, cur, lo, hi, nbits):
@@ -350,6 +371,28 @@ def _pins_hold(o):
         if int(np.frombuffer(sc[40:48].tobytes(), "<u8")[0]) <= int(np.frombuffer(s[40:48].tobytes(), "<u8")[0]):
             return False
         if not np.array_equal(o.recover(base, [sc]).view(np.uint32), once.view(np.uint32)):
+            return False
+        # mean representatives: hand cases (a tie to even, a third of an ulp, a negative bucket), then a stream whose
+        # representatives are the exact means of the deltas of each symbol
+        f1, fu = np.float32(1.0), np.float32(2.0 ** -23)
+        if o.bucket_mean([f1 + fu, f1 + 2 * fu]) != f1 + 2 * fu or o.bucket_mean([f1, f1 + fu]) != f1:
+            return False
+        if o.bucket_mean([f1 + fu, f1 + 2 * fu, f1 + 2 * fu]) != f1 + 2 * fu or o.bucket_mean([-3.0, -2.0]) != np.float32(-2.5):
+            return False
+        sm = o.compress_mean(base, cur, 3)
+        if sm[7] != 8:
+            return False
+        tabm = np.frombuffer(sm[64:64 + 16 * nsym].tobytes(), dtype=[("key", "<u2"), ("len", "u1"), ("pad", "u1"), ("rep", "<f4"), ("count", "<u8")])
+        tabp = np.frombuffer(s[64:64 + 16 * nsym].tobytes(), dtype=[("key", "<u2"), ("len", "u1"), ("pad", "u1"), ("rep", "<f4"), ("count", "<u8")])
+        changed = 0
+        for j in range(1, nsym):
+            dbits = d.astype(np.float32).view(np.uint32)
+            dkey = (dbits >> 31) * 256 + ((dbits >> 23) & 255)
+            vals = d[dkey == int(tabp["key"][j])].astype(np.float64)  # the deltas of symbol j
+            if vals.size != int(tabm["count"][j]) or abs(float(tabm["rep"][j]) - vals.mean()) > 2.0 ** -24 * abs(vals.mean()):
+                return False
+            changed += int(tabm["rep"][j] != tabp["rep"][j])
+        if changed == 0:
             return False
         # the threaded timing mode writes the same bytes and states
         if o.compress_mt(base, cur, 3, 3).tobytes() != s.tobytes():

@@ -415,7 +415,7 @@ def test_reader_rejects_corruption(oracle):
     expect(setb(0, ord("X")), oracle.ERR_FORMAT)     # magic
     expect(setb(4, 2), oracle.ERR_FORMAT)            # version
     expect(setb(6, 10), oracle.ERR_FORMAT)           # nbits
-    expect(setb(7, 8), oracle.ERR_FORMAT)            # flags
+    expect(setb(7, 16), oracle.ERR_FORMAT)           # flags
     expect(setb(16, 200), oracle.ERR_FORMAT)         # nsym > 2^nbits
     expect(setb(24, 1), oracle.ERR_FORMAT)           # chunk_elems
     expect(setb(64 + 16 + 2, 1), oracle.ERR_FORMAT)  # a code length changed: Kraft / payload_bits
@@ -780,5 +780,93 @@ def test_cached_stream_properties(oracle):
     # the cached-lengths flag goes with neither fixed-width codes nor shards
     bad = s2.copy()
     bad[7] = 5
+    with pytest.raises(oracle.OracleError):
+        oracle.recover(base, [bad])
+
+
+# ---- variant: bucket mean as the representative (format section 1.8) ------------------------------------------
+
+
+def _nearest_f32(x):
+    """fp32 value nearest to the exact rational x, ties to the even mantissa (by exact comparison of candidates)."""
+    from fractions import Fraction
+
+    c = np.float32(float(x))
+    cands = {np.float32(c), np.nextafter(c, np.float32(np.inf)), np.nextafter(c, np.float32(-np.inf))}
+    best = None
+    for v in cands:
+        dist = abs(Fraction(float(v)) - x)
+        even = (int(np.float32(v).view(np.uint32)) & 1) == 0
+        key = (dist, 0 if even else 1)
+        if best is None or key < best[0]:
+            best = (key, v)
+    return np.float32(best[1])
+
+
+def test_bucket_mean_hand_cases_and_exact_rational(oracle):
+    from fractions import Fraction
+
+    one = np.float32(1.0)
+    ulp = np.float32(2.0 ** -23)
+    assert oracle.bucket_mean([1.0, 1.25, 1.5]) == np.float32(1.25)
+    assert oracle.bucket_mean([one, one + ulp]) == one                           # tie: even mantissa 0
+    assert oracle.bucket_mean([one + ulp, one + 2 * ulp]) == one + 2 * ulp       # tie: even mantissa 2
+    assert oracle.bucket_mean([one + ulp, one + ulp, one + 2 * ulp]) == one + ulp  # 1 + 4/3 ulp
+    assert oracle.bucket_mean([one + ulp, one + 2 * ulp, one + 2 * ulp]) == one + 2 * ulp  # 1 + 5/3 ulp
+    assert oracle.bucket_mean([-3.0, -2.0]) == np.float32(-2.5)
+    assert oracle.bucket_mean([1.75]) == np.float32(1.75)
+    fmax = np.finfo(np.float32).max
+    assert oracle.bucket_mean([fmax, fmax, fmax]) == fmax                        # largest binade, no carry
+    tiny = np.float32(2.0 ** -126)
+    assert oracle.bucket_mean([tiny, tiny * np.float32(1.5)]) == tiny * np.float32(1.25)  # smallest normal binade
+    assert np.isnan(oracle.bucket_mean([1.0, 2.0]))                              # not one bucket
+    rng = np.random.default_rng(5)
+    for _ in range(300):
+        e = int(rng.integers(-120, 120))
+        k = int(rng.integers(1, 40))
+        sig = rng.integers(2 ** 23, 2 ** 24, k)
+        if rng.random() < 0.3:
+            sig = sig[0] + rng.integers(0, 3, k)  # values a few ulps apart: ties are frequent
+            sig = np.minimum(sig, 2 ** 24 - 1)
+        sign = -1.0 if rng.random() < 0.5 else 1.0
+        vals = (sign * sig.astype(np.float64) * 2.0 ** (e - 23)).astype(np.float32)
+        exact = sum(Fraction(float(v)) for v in vals) / k
+        assert oracle.bucket_mean(vals) == _nearest_f32(exact)
+
+
+def test_mean_stream_differs_from_the_plain_one_in_representatives_only(oracle):
+    rng = np.random.default_rng(77)
+    n, nbits = 2 * 4096 + 300, 3
+    base, cur = _random_case(rng, n)
+    plain, mean = oracle.compress(base, cur, nbits), oracle.compress_mean(base, cur, nbits)
+    p, q = _parse(plain), _parse(mean)
+    assert q["flags"] == 8 and p["flags"] == 0
+    for f in ("key", "len", "count"):
+        assert np.array_equal(p["tab"][f], q["tab"][f])
+    same = mean.copy()
+    same[7] = 0
+    same[64:64 + 16 * q["nsym"]] = plain[64:64 + 16 * p["nsym"]]
+    assert same.tobytes() == plain.tobytes()  # header flag and table apart, the same bytes
+    # every representative is the rounded exact mean of its bucket's deltas
+    d = (cur - base).astype(np.float32)
+    sym = oracle.symbols(base, cur, nbits)
+    reps = q["tab"]["rep"].view(np.float32)
+    from fractions import Fraction
+
+    for j in range(1, q["nsym"]):
+        vals = d[sym == j]
+        assert vals.size == int(q["tab"]["count"][j])
+        assert reps[j] == _nearest_f32(sum(Fraction(float(v)) for v in vals) / vals.size)
+    assert reps[0] == 0
+    # recovery adds those representatives; the squared error inside the kept buckets is not above the midrange's
+    out_mean, out_plain = oracle.recover(base, [mean]), oracle.recover(base, [plain])
+    assert np.array_equal(out_mean.view(np.uint32), (base + reps[sym]).astype(np.float32).view(np.uint32))
+    kept = sym > 0
+    err_mean = np.sum((out_mean.astype(np.float64) - cur)[kept] ** 2)
+    err_plain = np.sum((out_plain.astype(np.float64) - cur)[kept] ** 2)
+    assert err_mean <= err_plain * (1 + 1e-6)
+    # the flag goes alone
+    bad = mean.copy()
+    bad[7] = 9
     with pytest.raises(oracle.OracleError):
         oracle.recover(base, [bad])
