@@ -489,6 +489,19 @@ def run_ours(args, rank, world, local_rank):
               "bytes_vs_plain": int(info_c.total_bytes) / stream_bytes[-1]}
     del cache
 
+    # ---- variant: bucket means as representatives (LC_OPT_MEAN_REP); outside the timed region
+    mr = []
+    for it in range(4):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        lc.compress_opt_async(tracked, u, nbits, sbuf, ws, lc.OPT_MEAN_REP)
+        b.record()
+        torch.cuda.synchronize()
+        if it >= 1:
+            mr.append(a.elapsed_time(b))
+    assert lc.last_status(ws) == 0 and lc.stream_info(sbuf).mean_rep == 1
+    mean_rep = {"ms": statistics.median(mr)}
+
     # ---- per-layer granularity on the workload that has layers (ResNet-18-sized: 62 segments): one stream per
     # segment against one stream for the flat vector; outside the timed region
     per_layer = None
@@ -600,6 +613,7 @@ def run_ours(args, rank, world, local_rank):
                             "frac_of_peak": (12.0 * n + stream_bytes[-1]) / (cu_ms * 1e-3) / 1e9 / peak},
         "table_caching": cached,
         "per_layer": per_layer,
+        "mean_rep": mean_rep,
         # algorithmic bytes of a merge: read base and the chain's streams, write the merged stream
         "merge": None if merge_ms is None else {
             "ms": merge_ms, "streams_in": chain, "merged_ratio": 4.0 * n / merged_bytes,

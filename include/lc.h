@@ -58,6 +58,7 @@ typedef struct lc_info {
   uint32_t fixed_width;    /* 1 if the stream carries fixed-width codes (format section 1.5) */
   uint32_t shard;          /* 1 if the stream is a shard's, coded with the table of a larger vector (section 1.6) */
   uint32_t cached_lengths; /* 1 if the code lengths came from a length cache (format section 1.7) */
+  uint32_t mean_rep;       /* 1 if the representatives are bucket means (format section 1.8) */
 } lc_info;
 
 /* Library version (major*100 + minor). */
@@ -126,10 +127,18 @@ int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbit
  *               Huffman codes (format section 1.5): the stream of Section 3.1.1's size model, n*ceil(log2 k) bits
  *               of indices, and the "E" (with nbits 9) and "E+P" stages of Section 4.3's size breakdown as real
  *               streams. lc_recover reads such streams like any other. This option does change the bytes.
+ *               LC_OPT_MEAN_REP: a bucket is represented by the mean of its values, rounded once to fp32, instead
+ *               of the average of its maximum and minimum that Section 3.1.1 prescribes (format section 1.8). A
+ *               variant, not the paper's method: the mean minimises the squared error inside a bucket. Symbols,
+ *               code and payload are unchanged; only the table's representatives (and so the recovered values)
+ *               differ. The statistics pass then also sums the mantissas, exactly and in integers, so the result
+ *               is as deterministic as the default; that pass runs about 1.5 times as long. Not together with
+ *               LC_OPT_FIXED_WIDTH (LC_ERR_ARG).
  * Any other bit in `options` returns LC_ERR_ARG.
  */
 #define LC_OPT_NO_DEVICE_WAIT 1u
 #define LC_OPT_FIXED_WIDTH 2u
+#define LC_OPT_MEAN_REP 4u
 int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                     uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
                     uint32_t options, lc_cuda_stream_t cs);

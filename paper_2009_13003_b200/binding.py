@@ -31,7 +31,7 @@ class LCInfo(C.Structure):
         ("n", C.c_uint64), ("total_bytes", C.c_uint64), ("payload_bits", C.c_uint64),
         ("payload_offset", C.c_uint64), ("nbits", C.c_uint32), ("nsym", C.c_uint32),
         ("max_len", C.c_uint32), ("nchunks", C.c_uint32), ("valid", C.c_int32), ("fixed_width", C.c_uint32), ("shard", C.c_uint32),
-        ("cached_lengths", C.c_uint32),
+        ("cached_lengths", C.c_uint32), ("mean_rep", C.c_uint32),
     ]
 
 
@@ -147,6 +147,7 @@ def compress_update_async(base, cur, nbits, stream, tracked_out, workspace):
 
 OPT_NO_DEVICE_WAIT = 1
 OPT_FIXED_WIDTH = 2
+OPT_MEAN_REP = 4
 
 
 def compress_opt_async(base, cur, nbits, stream, workspace, options, tracked_out=None):
@@ -185,16 +186,17 @@ def stream_info(stream) -> LCInfo:
     return info
 
 
-def compress(base, cur, nbits, stream=None, workspace=None, fixed=False):
+def compress(base, cur, nbits, stream=None, workspace=None, fixed=False, mean=False):
     """stream <- LC(cur - base). Returns the stream trimmed to its size (a view of ``stream``). ``fixed``: fixed-width
-    bucket indices instead of the Huffman code (LC_OPT_FIXED_WIDTH)."""
+    bucket indices instead of the Huffman code (LC_OPT_FIXED_WIDTH). ``mean``: bucket means as representatives
+    (LC_OPT_MEAN_REP)."""
     n = base.numel()
     if stream is None:
         stream = alloc_stream(n, nbits, base.device)
     if workspace is None:
         workspace = alloc_workspace(n, base.device)
-    if fixed:
-        compress_opt_async(base, cur, nbits, stream, workspace, OPT_FIXED_WIDTH)
+    if fixed or mean:
+        compress_opt_async(base, cur, nbits, stream, workspace, (OPT_FIXED_WIDTH if fixed else 0) | (OPT_MEAN_REP if mean else 0))
     else:
         compress_async(base, cur, nbits, stream, workspace)
     _check(last_status(workspace), "lc_compress (device)")

@@ -43,8 +43,10 @@ int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, vo
   const uint64_t skip = keep_status ? sizeof(int32_t) : 0;
   cudaError_t e = cudaMemsetAsync(static_cast<uint8_t*>(workspace) + skip, 0, W.plane_off - skip, cs);
   if (e != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs)) != cudaSuccess) return LC_ERR_CUDA;
-  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, opt.fixed_width, nullptr, opt.length_cache, cs)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_stats(base, cur, n, c.ctl, c.plane, cs, opt.mean_rep)) != cudaSuccess) return LC_ERR_CUDA;
+  if ((e = launch_table(c.ctl, n, nbits, static_cast<uint8_t*>(stream), true, opt.fixed_width, nullptr, opt.length_cache, cs,
+                        opt.mean_rep)) != cudaSuccess)
+    return LC_ERR_CUDA;
   if ((e = launch_encode(c.ctl, c.tiles, c.plane, base, cur, n, static_cast<uint8_t*>(stream), tracked_out, opt,
                          cs)) != cudaSuccess)
     return LC_ERR_CUDA;
@@ -105,7 +107,8 @@ int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbit
 int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, void* stream,
                     uint64_t stream_capacity, float* tracked_out, void* workspace, uint64_t workspace_bytes,
                     uint32_t options, lc_cuda_stream_t cs) {
-  if (options & ~(uint32_t)(LC_OPT_NO_DEVICE_WAIT | LC_OPT_FIXED_WIDTH)) return LC_ERR_ARG;
+  if (options & ~(uint32_t)(LC_OPT_NO_DEVICE_WAIT | LC_OPT_FIXED_WIDTH | LC_OPT_MEAN_REP)) return LC_ERR_ARG;
+  if ((options & LC_OPT_MEAN_REP) && (options & LC_OPT_FIXED_WIDTH)) return LC_ERR_ARG;
   if (tracked_out) {
     const int rc = check_tracked_out(cur, n, tracked_out);
     if (rc != LC_OK) return rc;
@@ -113,6 +116,7 @@ int lc_compress_opt(const float* base, const float* cur, uint64_t n, int nbits, 
   EncodeOptions opt;
   opt.two_pass_scan = (options & LC_OPT_NO_DEVICE_WAIT) != 0;
   opt.fixed_width = (options & LC_OPT_FIXED_WIDTH) != 0;
+  opt.mean_rep = (options & LC_OPT_MEAN_REP) != 0;
   return compress_impl(base, cur, n, nbits, stream, stream_capacity, tracked_out, workspace, workspace_bytes, opt, cs);
 }
 
@@ -363,6 +367,7 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
   info->fixed_width = h[7] & 1u;
   info->shard = (h[7] >> 1) & 1u;
   info->cached_lengths = (h[7] >> 2) & 1u;
+  info->mean_rep = (h[7] >> 3) & 1u;
   info->n = le(8, 8);
   info->nsym = (uint32_t)le(16, 4);
   info->max_len = (uint32_t)le(20, 4);
@@ -370,7 +375,7 @@ int lc_stream_info(const void* stream, lc_info* info, lc_cuda_stream_t cs) {
   info->payload_bits = le(40, 8);
   info->total_bytes = le(48, 8);
   info->payload_offset = le(56, 8);
-  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 && h[7] <= 4 &&
+  info->valid = (h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1' && le(4, 2) == 1 && (h[7] <= 4 || h[7] == 8) &&
                  le(24, 4) == kChunkElems && le(28, 2) == kLanes && le(30, 2) == kGroup &&
                  le(36, 4) == kPayloadAlign)
                     ? 1

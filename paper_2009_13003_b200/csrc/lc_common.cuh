@@ -79,6 +79,7 @@ struct Control {
   uint32_t inv_min[kKeys];          // max over the bucket of ~bits (zero-initialised running minimum)
   uint32_t max_bits[kKeys];         // max over the bucket of bits
   EncEntry enc[kKeys];
+  unsigned long long mant_sum[kKeys];  // mean-representative variant only: sum of the bucket's mantissa fields
 };
 // The bucket statistics as a shard of a split vector hands them out and takes them back (include/lc.h, lc_shard_*):
 // the three arrays of Control, in Control's order, so that one copy moves them.
@@ -133,6 +134,7 @@ struct EncodeOptions {
   uint32_t spin_limit = 1u << 20; // polls of the look-back before it gives up with LC_ERR_TIMEOUT
   uint32_t ticket_bias = 0;       // added to every tile ticket (test aid: with 1, tile 0 is never coded)
   bool fixed_width = false;       // fixed-width codes (format section 1.5) instead of the Huffman code
+  bool mean_rep = false;          // bucket means as representatives (format section 1.8) instead of the midrange
   uint8_t* length_cache = nullptr;  // DEVICE, kLengthCacheBytes: code lengths of earlier calls (format section 1.7)
 };
 
@@ -140,15 +142,16 @@ constexpr uint32_t kLengthCacheRow = 512;                            // bytes pe
 constexpr uint64_t kLengthCacheBytes = 512ull * kLengthCacheRow;
 
 // ---- launchers (each defined next to its kernel) ---------------------------------------------------
+// mean: also accumulate the mantissa sums the mean-representative variant needs (a slower kernel variant)
 cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
-                         cudaStream_t cs);
+                         cudaStream_t cs, bool mean = false);
 // wide_ok: false if the encode pass will not be able to read base and cur (the table pass then rejects a vector
 // with an exponent field >= 128 with LC_ERR_RANGE)
 // fixed: fixed-width codes (format section 1.5) instead of the Huffman code
 // whole: nullptr, or the statistics of the whole vector of which this call codes a shard (format section 1.6):
 //        kept buckets, representatives and code then come from them, the table's counts from ctl's own
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, bool fixed,
-                         const ShardStats* whole, uint8_t* length_cache, cudaStream_t cs);
+                         const ShardStats* whole, uint8_t* length_cache, cudaStream_t cs, bool mean = false);
 // tracked_out: nullptr, or where to write base + quantized delta (may be base itself)
 cudaError_t launch_encode(Control* ctl, unsigned long long* tiles, const uint8_t* plane, const float* base,
                           const float* cur, uint64_t n, uint8_t* stream, float* tracked_out, const EncodeOptions& opt,

@@ -125,7 +125,7 @@ __device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8
       const bool magic = h[0] == 'L' && h[1] == 'C' && h[2] == 'C' && h[3] == '1';
       S.fixed = h[7] & 1u;
       S.shared_table = (h[7] >> 1) & 1u;
-      if (!magic || load_le(h + 4, 2) != 1 || nbits < 1 || nbits > (uint32_t)kMaxNbits || h[7] > 4) err = LC_ERR_FORMAT;  // bit 2 (cached lengths) goes alone
+      if (!magic || load_le(h + 4, 2) != 1 || nbits < 1 || nbits > (uint32_t)kMaxNbits || (h[7] > 4 && h[7] != 8)) err = LC_ERR_FORMAT;  // bits 2 (cached lengths) and 3 (mean) go alone
       else if (S.nsym < 1 || S.nsym > (1u << nbits) || S.max_len > 63) err = LC_ERR_FORMAT;
       else if (load_le(h + 24, 4) != kChunkElems || load_le(h + 28, 2) != kLanes ||
                load_le(h + 30, 2) != kGroup || load_le(h + 36, 4) != kPayloadAlign) err = LC_ERR_FORMAT;

@@ -32,6 +32,11 @@ constexpr int kStatsThreads = 384;
 constexpr int kRows = 8;  // steps per unit
 constexpr uint32_t kCntWords = kKeys * 32;
 constexpr uint32_t kStatsSmem = (kCntWords + 2 * kKeys) * 4;  // 64 KB + 4 KB
+// Mean-representative variant (format section 1.8): two more tables of the same shape hold, per key and lane, the
+// sums of the low 12 and of the high 11 bits of the mantissa fields. A column receives at most 32 elements per warp
+// and unit, so 32-bit sums hold for kMeanMaxUnitsPerWarp units per warp: 12 warps * 32 * 4095 * 2731 < 2^32.
+constexpr uint32_t kStatsSmemMean = (3 * kCntWords + 2 * kKeys) * 4;  // 192 KB + 4 KB: one CTA per SM
+constexpr uint64_t kMeanMaxUnitsPerWarp = 2731;
 
 __device__ __forceinline__ float4 ld_stream(const float4* p) {
   float4 v;
@@ -48,9 +53,16 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) {
 __device__ __forceinline__ uint32_t slot_of(uint32_t bits) { return ((bits >> 22) & 0x1FEu) | (bits >> 31); }
 __device__ __forceinline__ uint32_t key_of_slot(uint32_t slot) { return ((slot & 1u) << 8) | (slot >> 1); }
 
+template <bool MEAN>
 struct Acc {
   uint32_t* cnt_lane;  // &cnt[lane]
   uint2* mm;
+  __device__ __forceinline__ void sum(uint32_t bits, uint32_t slot) {
+    if (MEAN) {
+      atomicAdd(cnt_lane + kCntWords + slot * 32, bits & 0xFFFu);
+      atomicAdd(cnt_lane + 2 * kCntWords + slot * 32, (bits >> 12) & 0x7FFu);
+    }
+  }
   __device__ __forceinline__ void improve(uint32_t bits, uint32_t slot, uint2 cur) {
     if (~bits > cur.x) atomicMax(&mm[slot].x, ~bits);
     if (bits > cur.y) atomicMax(&mm[slot].y, bits);
@@ -58,6 +70,7 @@ struct Acc {
   __device__ __forceinline__ void add(uint32_t bits) {
     const uint32_t slot = slot_of(bits);
     atomicAdd(cnt_lane + slot * 32, 1u);
+    sum(bits, slot);
     improve(bits, slot, mm[slot]);
   }
   // Four elements at once: the four reads of the running min / max pairs go out together, and one test
@@ -69,6 +82,10 @@ struct Acc {
     atomicAdd(cnt_lane + k1 * 32, 1u);
     atomicAdd(cnt_lane + k2 * 32, 1u);
     atomicAdd(cnt_lane + k3 * 32, 1u);
+    sum(d0, k0);
+    sum(d1, k1);
+    sum(d2, k2);
+    sum(d3, k3);
     const bool any = (~d0 > c0.x) | (d0 > c0.y) | (~d1 > c1.x) | (d1 > c1.y) | (~d2 > c2.x) | (d2 > c2.y) |
                      (~d3 > c3.x) | (d3 > c3.y);
     if (any) {
@@ -80,19 +97,22 @@ struct Acc {
   }
 };
 
-__global__ void __launch_bounds__(kStatsThreads, 2)
+template <bool MEAN>
+__global__ void __launch_bounds__(kStatsThreads, MEAN ? 1 : 2)
 stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint64_t n, uint64_t nunits,
              Control* __restrict__ ctl, uint8_t* __restrict__ plane) {
   extern __shared__ __align__(16) uint32_t smem[];
+  // MEAN: cnt, then the two sum tables, then mm
+  constexpr uint32_t kTables = MEAN ? 3 : 1;
   uint32_t* cnt = smem;
-  uint2* mm = reinterpret_cast<uint2*>(smem + kCntWords);
-  for (uint32_t i = threadIdx.x; i < kCntWords + 2 * kKeys; i += kStatsThreads) smem[i] = 0;
+  uint2* mm = reinterpret_cast<uint2*>(smem + kTables * kCntWords);
+  for (uint32_t i = threadIdx.x; i < kTables * kCntWords + 2 * kKeys; i += kStatsThreads) smem[i] = 0;
   __syncthreads();
 
   const uint32_t lane = threadIdx.x & 31;
   const uint64_t warp = (uint64_t)blockIdx.x * (kStatsThreads / 32) + (threadIdx.x >> 5);
   const uint64_t nwarps = (uint64_t)gridDim.x * (kStatsThreads / 32);
-  Acc acc{cnt + lane, mm};
+  Acc<MEAN> acc{cnt + lane, mm};
 
   for (uint64_t u = warp; u < nunits; u += nwarps) {
     const uint64_t i0 = u * kUnitElems;
@@ -152,6 +172,14 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
       atomicAdd(&ctl->count[key], (unsigned long long)total);
       atomicMax(&ctl->inv_min[key], mm[slot].x);
       atomicMax(&ctl->max_bits[key], mm[slot].y);
+      if (MEAN) {
+        unsigned long long lo = 0, hi = 0;
+        for (uint32_t l = 0; l < 32; ++l) {
+          lo += cnt[kCntWords + slot * 32 + ((l + threadIdx.x) & 31)];
+          hi += cnt[2 * kCntWords + slot * 32 + ((l + threadIdx.x) & 31)];
+        }
+        atomicAdd(&ctl->mant_sum[key], lo + (hi << 12));
+      }
     }
   }
 }
@@ -159,33 +187,44 @@ stats_kernel(const float* __restrict__ base, const float* __restrict__ cur, uint
 }  // namespace
 
 cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
-                         cudaStream_t cs) {
+                         cudaStream_t cs, bool mean) {
   const WorkspaceLayout W = workspace_layout(n);
   if (W.nunits == 0) return cudaSuccess;
-  static int blocks_per_sm[kMaxDevices] = {}, sms[kMaxDevices] = {};  // by device ordinal
+  static int blocks_per_sm[kMaxDevices][2] = {}, sms[kMaxDevices] = {};  // by device ordinal and kernel variant
   const int dev = current_device_index();
   if (dev < 0) return cudaErrorInvalidDevice;
-  if (blocks_per_sm[dev] == 0) {
-    cudaError_t e = cudaFuncSetAttribute(stats_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmem);
+  const int v = mean ? 1 : 0;
+  const uint32_t smem = mean ? kStatsSmemMean : kStatsSmem;
+  const void* fn = mean ? reinterpret_cast<const void*>(stats_kernel<true>) : reinterpret_cast<const void*>(stats_kernel<false>);
+  if (blocks_per_sm[dev][v] == 0) {
+    cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     int nsm = 0;
     if ((e = cudaDeviceGetAttribute(&nsm, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     int bps = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, stats_kernel, kStatsThreads, kStatsSmem);
+    e = mean ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, stats_kernel<true>, kStatsThreads, smem)
+             : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bps, stats_kernel<false>, kStatsThreads, smem);
     if (e != cudaSuccess) return e;
     if (bps < 1) bps = 1;
     // carve-out in percent of the SM's 228 KB: the resident CTAs' shared memory (plus 1 KB each that the system
     // reserves), rounded up
-    const int carve = (int)(((uint64_t)bps * (kStatsSmem + 1024) * 100 + 228 * 1024 - 1) / (228 * 1024)) + 1;
-    e = cudaFuncSetAttribute(stats_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, carve < 100 ? carve : 100);
+    const int carve = (int)(((uint64_t)bps * (smem + 1024) * 100 + 228 * 1024 - 1) / (228 * 1024)) + 1;
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, carve < 100 ? carve : 100);
     if (e != cudaSuccess) return e;
     sms[dev] = nsm;
-    blocks_per_sm[dev] = bps;
+    blocks_per_sm[dev][v] = bps;
   }
   const uint64_t want = (W.nunits + kStatsThreads / 32 - 1) / (kStatsThreads / 32);
-  const uint64_t full = (uint64_t)sms[dev] * blocks_per_sm[dev];
+  const uint64_t full = (uint64_t)sms[dev] * blocks_per_sm[dev][v];
   const unsigned grid = (unsigned)(want < full ? want : full);
-  stats_kernel<<<grid, kStatsThreads, kStatsSmem, cs>>>(base, cur, n, W.nunits, ctl, plane);
+  if (mean) {
+    // the 32-bit column sums of the variant hold for a bounded number of units per warp (see kMeanMaxUnitsPerWarp)
+    const uint64_t nwarps = (uint64_t)grid * (kStatsThreads / 32);
+    if ((W.nunits + nwarps - 1) / nwarps > kMeanMaxUnitsPerWarp) return cudaErrorInvalidConfiguration;
+    stats_kernel<true><<<grid, kStatsThreads, smem, cs>>>(base, cur, n, W.nunits, ctl, plane);
+  } else {
+    stats_kernel<false><<<grid, kStatsThreads, smem, cs>>>(base, cur, n, W.nunits, ctl, plane);
+  }
   return cudaGetLastError();
 }
 

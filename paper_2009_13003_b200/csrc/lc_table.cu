@@ -21,7 +21,7 @@ __device__ __forceinline__ void store_le(uint8_t* p, uint64_t v, int bytes) {
 
 __global__ void __launch_bounds__(kTableThreads)
 table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restrict__ stream, int wide_ok,
-             int fixed, const ShardStats* __restrict__ whole, uint8_t* __restrict__ cache) {
+             int fixed, const ShardStats* __restrict__ whole, uint8_t* __restrict__ cache, int mean) {
   __shared__ uint32_t warp_cand[16];
   __shared__ uint16_t sym_of_key[kKeys];
   __shared__ unsigned long long sym_count[kMaxSym];
@@ -125,6 +125,15 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     const uint32_t t = mmin + mmax;
     uint32_t mr = t >> 1;
     if ((t & 1u) && (mr & 1u)) mr += 1;
+    if (mean) {
+      // variant (format section 1.8): mean of the mantissa fields, rounded to nearest, ties to even; it cannot reach
+      // 2^23 because it does not exceed the largest field
+      const unsigned long long sum = ctl->mant_sum[key];
+      unsigned long long q = sum / cnt;
+      const unsigned long long r = sum - q * cnt;
+      if (2 * r > cnt || (2 * r == cnt && (q & 1ull))) q += 1;
+      mr = (uint32_t)q;
+    }
     sym_rep[sym] = (key << 23) | mr;
     atomicAdd(&s_kept_total, cnt);
   }
@@ -285,7 +294,7 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
     h[0] = 'L'; h[1] = 'C'; h[2] = 'C'; h[3] = '1';
     store_le(h + 4, 1, 2);
     h[6] = (uint8_t)nbits;
-    h[7] = (uint8_t)((fixed ? 1 : 0) | (whole ? 2 : 0) | (hit ? 4 : 0));
+    h[7] = (uint8_t)((fixed ? 1 : 0) | (whole ? 2 : 0) | (hit ? 4 : 0) | (mean ? 8 : 0));
     store_le(h + 8, n, 8);
     store_le(h + 16, nsym, 4);
     store_le(h + 20, s_maxlen, 4);
@@ -309,8 +318,9 @@ table_kernel(Control* __restrict__ ctl, uint64_t n, int nbits, uint8_t* __restri
 }  // namespace
 
 cudaError_t launch_table(Control* ctl, uint64_t n, int nbits, uint8_t* stream, bool wide_ok, bool fixed,
-                         const ShardStats* whole, uint8_t* cache, cudaStream_t cs) {
-  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0, fixed ? 1 : 0, whole, cache);
+                         const ShardStats* whole, uint8_t* cache, cudaStream_t cs, bool mean) {
+  table_kernel<<<1, kTableThreads, 0, cs>>>(ctl, n, nbits, stream, wide_ok ? 1 : 0, fixed ? 1 : 0, whole, cache,
+                                            mean ? 1 : 0);
   return cudaGetLastError();
 }
 

@@ -53,7 +53,7 @@ def test_host_argument_checks_need_no_device():
     assert L.lc_compress_update(base, cur, 16, 4, stream, 8, 0x50000, ws, 1 << 20, None) == binding.ERR_CAPACITY
     assert L.lc_strerror(binding.ERR_FORMAT) == b"malformed stream"
     # lc_compress_opt: unknown option bits are refused before anything else happens
-    assert L.lc_compress_opt(base, cur, 16, 4, stream, 1 << 20, None, ws, 1 << 20, 4, None) == binding.ERR_ARG
+    assert L.lc_compress_opt(base, cur, 16, 4, stream, 1 << 20, None, ws, 1 << 20, 8, None) == binding.ERR_ARG
     assert L.lc_compress_opt(base, cur, 16, 4, stream, 1 << 20, cur, ws, 1 << 20, 1, None) == binding.ERR_ARG
 
 
