@@ -132,7 +132,7 @@ int lc_compress_update(const float* base, const float* cur, uint64_t n, int nbit
  *               variant, not the paper's method: the mean minimises the squared error inside a bucket. Symbols,
  *               code and payload are unchanged; only the table's representatives (and so the recovered values)
  *               differ. The statistics pass then also sums the mantissas, exactly and in integers, so the result
- *               is as deterministic as the default; that pass runs about 1.5 times as long. Not together with
+ *               is as deterministic as the default; that pass runs about 1.35 times as long. Not together with
  *               LC_OPT_FIXED_WIDTH (LC_ERR_ARG).
  * Any other bit in `options` returns LC_ERR_ARG.
  */

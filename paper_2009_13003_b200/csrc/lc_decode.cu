@@ -56,8 +56,9 @@ constexpr uint32_t kLongCode = 0x20000000u;
 template <int KS>
 constexpr int kPrefetchRows = KS == 1 ? 6 : 8;
 
-// The two lookup tables of a stream are 8 KB each and sit on 8 KB boundaries of shared memory.
+// The two lookup tables of a stream are 8 KB each; the first starts on a 128-byte boundary of shared memory.
 constexpr uint32_t kTableBytes = 8192;
+constexpr uint32_t kTablePad = 128;  // the tables start on a 128-byte boundary (a lane's copy of an entry is chosen by OR)
 static_assert((1 << kL1Bits) * kL1Rep * 8 == kTableBytes, "table sizes");
 
 struct alignas(16) StreamState {
@@ -428,13 +429,11 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
     asm volatile("prefetch.global.L2 [%0];" ::"l"(pf));
     pf = (j == kSteps - kPrefetchRows<KS> - 1) ? next_rows : pf + 128;
     int cnt0[KS];
-    uint32_t next0[KS];
     uint32_t flags = 0;
 #pragma unroll
     for (int s = 0; s < KS; ++s) {
-      cnt0[s] = bits[s].cnt;  // where the step starts, for the careful pass
-      next0[s] = bits[s].next;
       bits[s].refill(W[s]);
+      cnt0[s] = bits[s].cnt;  // where the step starts, for the careful pass (`next` does not move within a step)
     }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -469,7 +468,6 @@ __device__ __forceinline__ void decode_chunk_fast(const StreamState* S, const So
 #pragma unroll
         for (int s = 0; s < KS; ++s) {
           bits[s].cnt = cnt0[s];
-          bits[s].next = next0[s];
           bits[s].seek(W[s], bits[s].bitpos(W[s]));
         }
         // one element per trip; x is rotated so that the loop needs no indexed register
@@ -540,10 +538,10 @@ template <int KS>
 __global__ void __launch_bounds__(kDecMaxThreads, 1)
 decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, int32_t* __restrict__ status,
               const DecodeImage* __restrict__ images, uint32_t stage_bytes, uint64_t chunk_begin, uint64_t chunk_end) {
-  // dynamic shared memory: [pad to 8 KB | 2 tables per stream | StreamState per stream | staging areas]
+  // dynamic shared memory: [pad to 128 bytes | 2 tables per stream | StreamState per stream | staging areas]
   extern __shared__ __align__(16) unsigned char s_raw[];
-  unsigned char* tables = s_raw + ((kTableBytes - (smem_addr(s_raw) & (kTableBytes - 1))) & (kTableBytes - 1));
-  StreamState* S = reinterpret_cast<StreamState*>(s_raw + kTableBytes + KS * 2 * kTableBytes);
+  unsigned char* tables = s_raw + ((kTablePad - (smem_addr(s_raw) & (kTablePad - 1))) & (kTablePad - 1));
+  StreamState* S = reinterpret_cast<StreamState*>(s_raw + kTablePad + KS * 2 * kTableBytes);
   // the streams were validated and their tables built by decode_prepare_kernel: report a rejected stream (the same
   // words for every thread) or copy the images in
 #pragma unroll
@@ -660,7 +658,7 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
                              int32_t* status, const DecodeImage* images, uint64_t chunk_begin, uint64_t chunk_end,
                              cudaStream_t cs) {
   static int sms_of[kMaxDevices] = {};  // by device ordinal; non-zero once the kernel's attributes are set there
-  constexpr uint32_t kTables = kTableBytes + KS * (2 * kTableBytes + sizeof(StreamState));
+  constexpr uint32_t kTables = kTablePad + KS * (2 * kTableBytes + sizeof(StreamState));
   constexpr uint32_t kMaxDyn = kSmemPerSm - 1024 - kOverrunBytes;  // room for static __shared__ and the padding
   const int dev = current_device_index();
   if (dev < 0) return cudaErrorInvalidDevice;
