@@ -469,3 +469,33 @@ def test_host_buffer_entry_points(lc, oracle, n, k):
         with pytest.raises(Exception):
             lc.recover_host(bh, [sh[:size]] * (k - 1) + [bad], oh, arena)
         lc.recover_host(bh, [sh[:size]] * k, oh, arena)
+
+
+def test_more_than_2_31_elements(lc, oracle):
+    """A vector of 2^31 + 3 * 4096 + 5 elements (8.6 GB of fp32, ragged tail): every element index, chunk number and
+    byte offset beyond 32 bits' signed range. The stream is compared byte for byte with the oracle's (all host
+    cores), the recovered state bit for bit."""
+    from paper_2009_13003_b200 import synth
+
+    n, nbits = (1 << 31) + 3 * 4096 + 5, 4
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * (1 << 30):
+        pytest.skip("needs 40 GB of free device memory")
+    base = synth.normal(n, 0.02, DEV, 31)
+    cur = base + synth.laplace(n, 1e-3, DEV, 32)
+    ws, sbuf = lc.alloc_workspace(n, DEV), lc.alloc_stream(n, nbits, DEV)
+    lc.compress_async(base, cur, nbits, sbuf, ws)
+    assert lc.last_status(ws) == 0
+    info = lc.stream_info(sbuf)
+    assert info.valid == 1 and info.n == n and info.nchunks == (n + 4095) // 4096
+    base_h, cur_h = to_np(base), to_np(cur)
+    want = oracle.compress(base_h, cur_h, nbits, threads=ORACLE_THREADS)
+    assert want.size == info.total_bytes
+    got = to_np(sbuf[: info.total_bytes])
+    step = 1 << 28
+    for lo in range(0, want.size, step):
+        assert got[lo: lo + step].tobytes() == want[lo: lo + step].tobytes(), "stream differs near byte %d" % lo
+    del got, cur_h
+    out = lc.recover(base, [sbuf[: info.total_bytes]], out=cur, workspace=ws)  # cur is no longer needed
+    want_out = oracle.recover(base_h, [want], threads=ORACLE_THREADS)
+    assert np.array_equal(to_np(out).view(np.uint32), want_out.view(np.uint32))
