@@ -564,17 +564,37 @@ encode_kernel(Control* __restrict__ ctl, unsigned long long* __restrict__ tiles,
 constexpr int kScanThreads = 1024;
 
 // Size in bytes of every chunk (format section 3.3: the chunk's bits rounded up to 16 bytes), one warp per chunk,
-// into sizes[c].
+// into sizes[c]. Whole chunks whose keys the one-byte plane identifies take their code lengths from a 256-byte
+// table in shared memory, 16 plane bytes per load; the vector's partial last chunk and vectors with exponent
+// fields >= 128 go through the slow path's counting mode.
 __global__ void __launch_bounds__(kEncThreads)
 encode_sizes_kernel(const Control* __restrict__ ctl, unsigned long long* __restrict__ sizes,
                     const uint8_t* __restrict__ plane, const float* base, const float* __restrict__ cur, uint64_t n,
                     uint64_t nchunks) {
+  __shared__ uint8_t s_len[256];  // code length by plane byte (lengths are at most 63)
   if (ctl->status != 0) return;  // nothing in this kernel writes the word: the same for every thread
+  for (uint32_t b = threadIdx.x; b < 256; b += kEncThreads) s_len[b] = (uint8_t)ctl->enc[((b & 1u) << 8) | (b >> 1)].len;
+  __syncthreads();
   const uint32_t lane = threadIdx.x & 31;
   const KeySource ks{plane, base, cur, ctl->wide != 0};
   const uint64_t warp0 = (uint64_t)blockIdx.x * kEncWarps + (threadIdx.x >> 5), nwarps = (uint64_t)gridDim.x * kEncWarps;
   for (uint64_t c = warp0; c < nchunks; c += nwarps) {
-    uint32_t bits = chunk_slow(ctl->enc, ks, c, lane, n, nullptr, 0);
+    uint32_t bits = 0;
+    if (!ks.wide && (c + 1) * kChunkElems <= n) {
+      const uint4* ep = reinterpret_cast<const uint4*>(plane + c * kChunkElems) + lane;
+      uint4 v[kSteps / 4];
+#pragma unroll
+      for (uint32_t q = 0; q < kSteps / 4; ++q) v[q] = __ldg(ep + 32 * q);
+#pragma unroll
+      for (uint32_t q = 0; q < kSteps / 4; ++q) {
+        const uint32_t w[4] = {v[q].x, v[q].y, v[q].z, v[q].w};
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+          bits += s_len[w[r] & 255u] + s_len[(w[r] >> 8) & 255u] + s_len[(w[r] >> 16) & 255u] + s_len[w[r] >> 24];
+      }
+    } else {
+      bits = chunk_slow(ctl->enc, ks, c, lane, n, nullptr, 0);
+    }
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) bits += __shfl_xor_sync(0xffffffffu, bits, d);
     if (lane == 0) sizes[c] = align_up((bits + 7) / 8, kPayloadAlign);
