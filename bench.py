@@ -627,7 +627,8 @@ def run_ours(args, rank, world, local_rank):
                   "code_bits_per_element": code_bits, "entropy_bits_per_element": entropy_bits},
         "size_model": size_model,
         "roofline": roofline, "clocks": clocks, "e2e": e2e,
-        "gpu_launches": (3 + decode_launches) * args.steps,  # stats, table, encode + decode kernels per step
+        # per step: stats, table, encode; per group of up to four streams a prepare and a decode kernel
+        "gpu_launches": (3 + 2 * decode_launches) * args.steps,
     }
     if world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = oracle_baseline(cfg, n)
