@@ -38,6 +38,15 @@ int compress_impl(const float* base, const float* cur, uint64_t n, int nbits, vo
   if (workspace_bytes < W.total || stream_capacity < lc_stream_bound(n, nbits)) return LC_ERR_CAPACITY;
   const Carved c = carve(workspace, W);
 
+  // a small vector with the default options: one CTA does everything in one launch (no memset either)
+  if (n > 0 && n <= kSmallMaxElems && !opt.two_pass_scan && !opt.fixed_width && !opt.mean_rep && !opt.length_cache &&
+      opt.ticket_bias == 0 && opt.spin_limit == EncodeOptions().spin_limit) {
+    if (launch_small_compress(c.ctl, base, cur, n, nbits, static_cast<uint8_t*>(stream), tracked_out, keep_status, cs) !=
+        cudaSuccess)
+      return LC_ERR_CUDA;
+    return LC_OK;
+  }
+
   // control block and tile descriptors start at zero (keep_status: all but the status word, which holds the
   // outcome of the pass that produced `cur`; the table pass then leaves the vector alone if it is set)
   const uint64_t skip = keep_status ? sizeof(int32_t) : 0;

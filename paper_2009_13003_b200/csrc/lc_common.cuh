@@ -141,7 +141,13 @@ struct EncodeOptions {
 constexpr uint32_t kLengthCacheRow = 512;                            // bytes per row: one row per number of used symbols
 constexpr uint64_t kLengthCacheBytes = 512ull * kLengthCacheRow;
 
+// Vectors of at most this many elements (16 chunks) take the single-CTA, single-launch compress path.
+constexpr uint64_t kSmallMaxElems = 16 * kChunkElems;
+
 // ---- launchers (each defined next to its kernel) ---------------------------------------------------
+// the whole compress pass of a small vector (0 < n <= kSmallMaxElems) in one launch; tracked_out may be null
+cudaError_t launch_small_compress(Control* ctl, const float* base, const float* cur, uint64_t n, int nbits,
+                                  uint8_t* stream, float* tracked_out, bool keep_status, cudaStream_t cs);
 // mean: also accumulate the mantissa sums the mean-representative variant needs (a slower kernel variant)
 cudaError_t launch_stats(const float* base, const float* cur, uint64_t n, Control* ctl, uint8_t* plane,
                          cudaStream_t cs, bool mean = false);
