@@ -141,8 +141,10 @@ struct EncodeOptions {
 constexpr uint32_t kLengthCacheRow = 512;                            // bytes per row: one row per number of used symbols
 constexpr uint64_t kLengthCacheBytes = 512ull * kLengthCacheRow;
 
-// Vectors of at most this many elements (16 chunks) take the single-CTA, single-launch compress path.
-constexpr uint64_t kSmallMaxElems = 16 * kChunkElems;
+// Vectors of at most this many elements (one chunk) take the single-CTA, single-launch compress path. Measured per
+// call: 24 us at 64 elements, 30 us at 1000, 45 us at 4096, against 44-48 us for the memset and three launches of the
+// general path at any of these sizes; from two chunks on the general path is the faster one.
+constexpr uint64_t kSmallMaxElems = kChunkElems;
 
 // ---- launchers (each defined next to its kernel) ---------------------------------------------------
 // the whole compress pass of a small vector (0 < n <= kSmallMaxElems) in one launch; tracked_out may be null
