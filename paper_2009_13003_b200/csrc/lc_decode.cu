@@ -100,7 +100,7 @@ __device__ __forceinline__ uint2 canonical_lookup(const StreamState& S, uint32_t
 
 // Parses and validates stream `s`, then builds its decode tables in shared memory. All threads of the
 // CTA call this; returns 0 or the error to report.
-__device__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8_t* __restrict__ s,
+__device__ __noinline__ int prepare_stream(StreamState& S, unsigned char* tables, const uint8_t* __restrict__ s,
                               uint64_t bytes, uint64_t n, int* s_err) {
   const int tid = threadIdx.x, nthreads = blockDim.x;
   if (tid < 4 && bytes >= kHeaderBytes)
@@ -542,18 +542,30 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
   extern __shared__ __align__(16) unsigned char s_raw[];
   unsigned char* tables = s_raw + ((kTablePad - (smem_addr(s_raw) & (kTablePad - 1))) & (kTablePad - 1));
   StreamState* S = reinterpret_cast<StreamState*>(s_raw + kTablePad + KS * 2 * kTableBytes);
-  // the streams were validated and their tables built by decode_prepare_kernel: report a rejected stream (the same
-  // words for every thread) or copy the images in
+  // A launch of a single CTA (a vector of a few chunks) validates the streams and builds their tables itself, which
+  // saves the prepare kernel's launch; `images` is null then.
+  __shared__ int s_err;
+  if (images == nullptr) {
+    for (int s = 0; s < KS; ++s) {
+      const int err = prepare_stream(S[s], tables + s * 2 * kTableBytes, streams.ptr[s], streams.bytes[s], n, &s_err);
+      if (err) {  // the same value for every thread
+        if (threadIdx.x == 0) set_status(status, err);
+        return;
+      }
+    }
+  }
+  // otherwise the streams were validated and their tables built by decode_prepare_kernel: report a rejected stream
+  // (the same words for every thread) or copy the images in
 #pragma unroll
   for (int s = 0; s < KS; ++s) {
-    const int err = images[s].err;
+    const int err = images ? images[s].err : 0;
     if (err) {
       if (threadIdx.x == 0) set_status(status, err);
       return;
     }
   }
 #pragma unroll
-  for (int s = 0; s < KS; ++s) {
+  for (int s = 0; s < KS && images != nullptr; ++s) {
     uint2* l1 = reinterpret_cast<uint2*>(tables + s * 2 * kTableBytes);
     uint2* sub = l1 + kTableBytes / 8;
     const uint32_t sub_addr = smem_addr(sub);
@@ -655,8 +667,8 @@ decode_kernel(const float* base, DecodeStreams streams, uint64_t n, float* out, 
 
 template <int KS>
 cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, uint64_t n, float* out,
-                             int32_t* status, const DecodeImage* images, uint64_t chunk_begin, uint64_t chunk_end,
-                             cudaStream_t cs) {
+                             int32_t* status, DecodeImage* images, uint64_t chunk_begin, uint64_t chunk_end,
+                             bool prepare, cudaStream_t cs) {
   static int sms_of[kMaxDevices] = {};  // by device ordinal; non-zero once the kernel's attributes are set there
   constexpr uint32_t kTables = kTablePad + KS * (2 * kTableBytes + sizeof(StreamState));
   constexpr uint32_t kMaxDyn = kSmemPerSm - 1024 - kOverrunBytes;  // room for static __shared__ and the padding
@@ -734,7 +746,18 @@ cudaError_t launch_decode_ks(const float* base, const DecodeStreams& streams, ui
     if (cudaFuncSetAttribute(decode_kernel<KS>, cudaFuncAttributePreferredSharedMemoryCarveout, carve) != cudaSuccess)
       return cudaErrorUnknown;
   }
-  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, images, stage, chunk_begin, chunk_end);
+  // The streams' tables: built by one CTA per stream ahead of a launch of many CTAs, by the decoding CTA itself when
+  // there is only one (`images` null), or left from an earlier launch over the same streams (`prepare` false).
+  const DecodeImage* use = images;
+  if (prepare) {
+    if (grid == 1) {
+      use = nullptr;
+    } else {
+      decode_prepare_kernel<<<KS, kPrepThreads, kPrepSmem, cs>>>(streams, n, images);
+      if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
+    }
+  }
+  decode_kernel<KS><<<grid, warps * 32, dyn, cs>>>(base, streams, n, out, status, use, stage, chunk_begin, chunk_end);
   return cudaGetLastError();
 }
 
@@ -757,15 +780,11 @@ cudaError_t launch_decode(const float* base, const DecodeStreams& streams, int k
     prep_ready[dev] = true;
   }
   DecodeImage* img = static_cast<DecodeImage*>(images);
-  if (prepare) {
-    decode_prepare_kernel<<<k, kPrepThreads, kPrepSmem, cs>>>(streams, n, img);
-    if (cudaGetLastError() != cudaSuccess) return cudaErrorLaunchFailure;
-  }
   switch (k) {
-    case 1: return launch_decode_ks<1>(base, streams, n, out, status, img, chunk_begin, chunk_end, cs);
-    case 2: return launch_decode_ks<2>(base, streams, n, out, status, img, chunk_begin, chunk_end, cs);
-    case 3: return launch_decode_ks<3>(base, streams, n, out, status, img, chunk_begin, chunk_end, cs);
-    case 4: return launch_decode_ks<4>(base, streams, n, out, status, img, chunk_begin, chunk_end, cs);
+    case 1: return launch_decode_ks<1>(base, streams, n, out, status, img, chunk_begin, chunk_end, prepare, cs);
+    case 2: return launch_decode_ks<2>(base, streams, n, out, status, img, chunk_begin, chunk_end, prepare, cs);
+    case 3: return launch_decode_ks<3>(base, streams, n, out, status, img, chunk_begin, chunk_end, prepare, cs);
+    case 4: return launch_decode_ks<4>(base, streams, n, out, status, img, chunk_begin, chunk_end, prepare, cs);
     default: return cudaErrorInvalidValue;
   }
 }
